@@ -1,0 +1,192 @@
+/*
+ * flux_attn.h -- C ABI of libflux_attn.so: routed hybrid attention for one B200.
+ *
+ * The library runs the per-layer hot path of Flux Attention: a cached hard
+ * routing bit per (request, layer) sends the layer to causal Full Attention
+ * (Eq. 1) or to Sparse Attention over a condensed KV subset (Eq. 2; here the
+ * streaming subset: an attention sink of `sink` leading positions plus a local
+ * window of the `window` latest positions, query included), in prefill and in
+ * autoregressive decode.
+ *
+ * General rules
+ *  - Every entry point returns FLUX_OK (0) or a negative FLUX_E_* code; none
+ *    throws, exits or prints.  flux_last_error() gives a message for the last
+ *    failure on the calling thread.
+ *  - The library allocates no device memory.  The caller owns every device
+ *    buffer, including the workspace whose size flux_workspace_size() reports;
+ *    a plan owns host memory only.
+ *  - "device" pointers are CUDA global-memory addresses valid on the current
+ *    device; "host" pointers are ordinary CPU addresses.  Each argument says
+ *    which it is.  Device buffers must be 16-byte aligned.
+ *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL
+ *    for the default stream) unless stated otherwise.  Conditions that only the
+ *    device can see (a mask byte outside {0,1}, a NaN logit, a context length
+ *    outside [1, max_context], a wait that ran out) set bits in a device status
+ *    word; flux_plan_status() synchronises the stream and returns them.
+ *  - All tensors are bfloat16 unless stated otherwise; accumulation is fp32.
+ *  - Layouts: Q and O rows are [n_q_heads][head_dim]; a KV cache of one
+ *    (layer, request) is [rows][n_kv_heads][head_dim], token-major, so one
+ *    token's keys of all heads are one contiguous 2*n_kv_heads*head_dim-byte row.
+ *    Query head h reads KV head h / (n_q_heads / n_kv_heads).
+ *  - Mask encoding (Sec. 3.1, "Deterministic Inference via Hard Routing"):
+ *    1 = FA, 0 = SA.
+ */
+#ifndef FLUX_ATTN_H
+#define FLUX_ATTN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define FLUX_OK                   0
+#define FLUX_E_INVALID_ARG       -1  /* null / misaligned pointer, bad index, bad size          */
+#define FLUX_E_UNSUPPORTED_SHAPE -2  /* head_dim != 128, n_q_heads % n_kv_heads != 0, G > 16    */
+#define FLUX_E_CAPACITY          -3  /* batch or length beyond what the plan was created for    */
+#define FLUX_E_WORKSPACE         -4  /* workspace missing or too small                          */
+#define FLUX_E_DEVICE_TIMEOUT    -5  /* a bounded device-side wait gave up                      */
+#define FLUX_E_CUDA              -6  /* a CUDA runtime / driver call failed                     */
+#define FLUX_E_DEVICE_FLAG       -7  /* device-side input check failed (see status bits)        */
+
+/* bits of the device status word returned by flux_plan_status() */
+#define FLUX_STATUS_BAD_MASK      1u   /* mask byte not 0/1                                     */
+#define FLUX_STATUS_NAN_LOGIT     2u   /* routing logit is NaN                                  */
+#define FLUX_STATUS_BAD_LENGTH    4u   /* ctx_len / pos outside [1, max_context]                */
+#define FLUX_STATUS_WAIT_EXPIRED  8u   /* an mbarrier wait hit its iteration limit              */
+
+#define FLUX_KV_FULL        0  /* every layer's cache holds every position: row = position          */
+#define FLUX_KV_COMPACT_SA  1  /* an SA layer's cache holds sink + window rows only (Sec. 3.3)      */
+
+typedef struct {
+    int32_t n_layers;
+    int32_t n_q_heads;
+    int32_t n_kv_heads;
+    int32_t head_dim;       /* must be 128                                                      */
+    int32_t sink;           /* S >= 0: leading positions every SA query keeps                   */
+    int32_t window;         /* W >= 1: latest positions an SA query keeps, itself included      */
+    float   softmax_scale;  /* 0 selects 1/sqrt(head_dim); Eq. 1 leaves the scale out           */
+    int32_t max_batch;      /* largest B any call will pass                                     */
+    int32_t max_context;    /* largest context length; every full cache has >= this many rows   */
+    int32_t kv_layout;      /* FLUX_KV_FULL or FLUX_KV_COMPACT_SA                               */
+} flux_config;
+
+typedef struct flux_plan flux_plan; /* opaque host object */
+
+/* Plan life cycle.  Creating a plan validates the configuration and queries the
+ * current device (SM count, shared memory); it launches nothing.  Host memory
+ * only; flux_plan_destroy frees it.  *plan is set to NULL on failure. */
+int flux_plan_create(const flux_config *cfg, flux_plan **plan);
+int flux_plan_destroy(flux_plan *plan);
+
+/* Device workspace (split-K partials, status word, debug records, staging for
+ * the *_host calls).  bytes_out (host) receives the size for this configuration.
+ * The caller allocates it (256-byte aligned), zero-fills it once, and hands it
+ * over; it must stay valid and untouched by others while the plan is in use. */
+int flux_workspace_size(const flux_config *cfg, size_t *bytes_out);
+int flux_plan_set_workspace(flux_plan *plan, void *workspace /*device*/, size_t bytes);
+
+/* Hard routing, once per request batch at prefill; the result is cached for all
+ * decode steps (Sec. 3.1 "Deterministic Inference via Hard Routing", Sec. 3.3).
+ *   logits       fp32 [B][n_layers][2], FA logit first; device or host memory;
+ *                ignored when mask_or_null is given.
+ *   mask_or_null uint8 [B][n_layers] ready-made decisions (device or host), or NULL.
+ *   mask_out     uint8 [B][n_layers], device; receives 1 where pi_FA >= pi_SA (a tie
+ *                keeps FA), else 0.  The plan remembers this pointer: later calls
+ *                read the routing decision from it, so it must stay alive.
+ * Host inputs are validated on the host (NaN logit or mask byte outside {0,1}
+ * -> FLUX_E_INVALID_ARG, nothing launched) and staged through the workspace;
+ * device inputs are checked by the kernel (status bits).  B <= max_batch. */
+int flux_router_apply(flux_plan *plan, const float *logits, const uint8_t *mask_or_null,
+                      int32_t B, uint8_t *mask_out, void *stream);
+
+/* Prefill of one layer for one request (Eq. 1 or Eq. 2 by mask[req][layer]),
+ * causal.  Query rows sit at absolute positions q_start .. q_start+Nq-1 (chunked
+ * prefill, Appendix D.3 "chunk size"); k, v hold positions 0 .. q_start+Nq-1 as
+ * [rows][n_kv_heads][head_dim] with row = position (a FULL-layout cache or the
+ * projection output itself).
+ *   q, out   [Nq][n_q_heads][head_dim], device.    k, v  device, read only.
+ * Nq == 0 is a successful no-op.  q_start + Nq <= max_context. */
+int flux_attn_prefill(flux_plan *plan, int32_t layer, int32_t req, const void *q,
+                      const void *k, const void *v, int32_t q_start, int32_t Nq,
+                      void *out, void *stream);
+
+/* Sparse-decode KV retention after prefill (Sec. 3.3: a sparse layer keeps only
+ * the rows its kernel needs).  Copies, for one (layer, request), the rows of
+ * k_src/v_src ([n][n_kv_heads][head_dim], row = position) that decode will need
+ * into the layer's cache: all n rows for an FA layer or the FULL layout; for an
+ * SA layer in the COMPACT_SA layout rows [0,S) to slots [0,S) and rows
+ * [max(S,n-W), n) to slot S + ((position - S) mod W).  All pointers device. */
+int flux_kv_retain(flux_plan *plan, int32_t layer, int32_t req, const void *k_src,
+                   const void *v_src, int32_t n, void *k_cache, void *v_cache, void *stream);
+
+/* Append one new token per request to the caches of one layer (Sec. 3.3).
+ *   k_new, v_new       [B][n_kv_heads][head_dim], device.
+ *   k_caches, v_caches device arrays of B device pointers (this layer's cache of
+ *                      each request).
+ *   pos                int32 [B], device: position being written (= context length
+ *                      before the append).  pos < 0 skips the request.
+ * FA layers and the FULL layout write row pos; SA layers in COMPACT_SA write
+ * slot pos (pos < S) or S + ((pos - S) mod W). */
+int flux_kv_append(flux_plan *plan, int32_t layer, int32_t B, const void *k_new,
+                   const void *v_new, void *const *k_caches, void *const *v_caches,
+                   const int32_t *pos, void *stream);
+
+/* One decode step of one layer for the whole batch: one query row per request at
+ * position ctx_len-1 (its K, V already appended).  FA requests stream the whole
+ * cache, SA requests only sink + window rows (Appendix C.3, "fetches only the
+ * locally required KV"); one launch serves mixed modes, split over all SMs in
+ * equal-byte spans, followed by a combine pass.
+ *   q, out    [B][n_q_heads][head_dim], device.
+ *   k_caches, v_caches  device arrays of B device pointers.
+ *   ctx_len   int32 [B], device: context length including the new token;
+ *             <= 0 marks an inactive request (its output row is zero-filled). */
+int flux_attn_decode(flux_plan *plan, int32_t layer, int32_t B, const void *q,
+                     const void *const *k_caches, const void *const *v_caches,
+                     const int32_t *ctx_len, void *out, void *stream);
+
+/* The same decode step for callers whose activations live in host memory: copies
+ * q, k_new, v_new (host, pinned for speed) to staging in the workspace, appends,
+ * attends, and copies the result to out (host).  Asynchronous on `stream` like
+ * the rest; the host buffers must stay untouched until the stream is synchronised.
+ * The caches, pointer tables, pos and ctx_len stay on the device. */
+int flux_attn_decode_host(flux_plan *plan, int32_t layer, int32_t B, const void *q_host,
+                          const void *k_new_host, const void *v_new_host,
+                          void *const *k_caches, void *const *v_caches, const int32_t *pos,
+                          const int32_t *ctx_len, void *out_host, void *stream);
+
+/* Prefill for host-resident activations: q (host) is copied to the device buffer
+ * q_dev, the layer runs as flux_attn_prefill, and out_dev is copied to out_host. */
+int flux_attn_prefill_host(flux_plan *plan, int32_t layer, int32_t req, const void *q_host,
+                           void *q_dev, const void *k, const void *v, int32_t q_start,
+                           int32_t Nq, void *out_dev, void *out_host, void *stream);
+
+/* Synchronises `stream`, reads the device status word and clears it.  Returns
+ * FLUX_OK with *status_bits == 0, FLUX_E_DEVICE_TIMEOUT if a wait expired, or
+ * FLUX_E_DEVICE_FLAG for the input-check bits.  status_bits (host) may be NULL. */
+int flux_plan_status(flux_plan *plan, uint32_t *status_bits, void *stream);
+
+/* Dispatch record of the latest flux_attn_decode / flux_attn_prefill on this
+ * plan, for verification: synchronises `stream` and copies n_records records of
+ * 8 int32 each to records_out (host):
+ *   { mode (1 FA, 0 SA), layer, request, n, a_begin, a_end, b_begin, b_end }
+ * where [a_begin,a_end) and [b_begin,b_end) are the cache rows the kernel reads
+ * for the newest query row (b is empty for FA).  Decode writes one record per
+ * request, prefill one record.  n_records_out (host) receives the count. */
+int flux_debug_dispatch(flux_plan *plan, int32_t *records_out, int32_t max_records,
+                        int32_t *n_records_out, void *stream);
+
+/* Number of kernels this plan has launched so far (host counter). */
+int64_t flux_launch_count(const flux_plan *plan);
+
+/* Message for the most recent failure on the calling thread ("" if none). */
+const char *flux_last_error(void);
+
+/* Library version, "major.minor". */
+const char *flux_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FLUX_ATTN_H */

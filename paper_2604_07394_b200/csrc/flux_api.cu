@@ -1,0 +1,533 @@
+// Entry points of libflux_attn.so: plan, workspace, hard routing, KV append and
+// retention, status and dispatch records.  The attention kernels live in
+// flux_decode.cu and flux_prefill*.cu.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "flux_internal.h"
+
+namespace flux {
+
+static thread_local char g_err[512] = "";
+
+int fail(int code, const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+int check_cuda(cudaError_t e, const char *what)
+{
+    if (e == cudaSuccess) return FLUX_OK;
+    return fail(FLUX_E_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static int validate_config(const flux_config *c)
+{
+    if (!c) return fail(FLUX_E_INVALID_ARG, "config is NULL");
+    if (c->head_dim != kHeadDim)
+        return fail(FLUX_E_UNSUPPORTED_SHAPE, "head_dim %d unsupported (must be 128)", c->head_dim);
+    if (c->n_layers < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1)
+        return fail(FLUX_E_INVALID_ARG, "n_layers, n_q_heads, n_kv_heads must be >= 1");
+    if (c->n_q_heads % c->n_kv_heads != 0)
+        return fail(FLUX_E_UNSUPPORTED_SHAPE, "n_q_heads %d is not a multiple of n_kv_heads %d",
+                    c->n_q_heads, c->n_kv_heads);
+    if (c->n_q_heads / c->n_kv_heads > 16)
+        return fail(FLUX_E_UNSUPPORTED_SHAPE, "more than 16 query heads per KV head");
+    if (c->sink < 0 || c->window < 1)
+        return fail(FLUX_E_INVALID_ARG, "need sink >= 0 and window >= 1");
+    if (c->max_batch < 1 || c->max_batch > kMaxBatch)
+        return fail(FLUX_E_CAPACITY, "max_batch must be in [1, %d]", kMaxBatch);
+    if (c->max_context < 1 || (int64_t)c->max_context + 1 >= (1ll << 30))
+        return fail(FLUX_E_CAPACITY, "max_context must be in [1, 2^30)");
+    if ((int64_t)c->sink + c->window >= (1ll << 30))
+        return fail(FLUX_E_CAPACITY, "sink + window too large");
+    if (c->kv_layout != FLUX_KV_FULL && c->kv_layout != FLUX_KV_COMPACT_SA)
+        return fail(FLUX_E_INVALID_ARG, "unknown kv_layout %d", c->kv_layout);
+    if (!(c->softmax_scale >= 0.0f) || isinf(c->softmax_scale))
+        return fail(FLUX_E_INVALID_ARG, "softmax_scale must be finite and >= 0");
+    return FLUX_OK;
+}
+
+WorkspaceLayout workspace_layout(const flux_config &c)
+{
+    WorkspaceLayout w;
+    const size_t A = 256;
+    size_t off = 0;
+    const int G = c.n_q_heads / c.n_kv_heads;
+    const size_t B = (size_t)c.max_batch, L = (size_t)c.n_layers;
+    w.status = off;       off = align_up(off + 64, A);
+    w.debug = off;        off = align_up(off + B * 8 * sizeof(int32_t), A);
+    w.sched = off;        off = align_up(off + (B + 4) * sizeof(int32_t), A);
+    w.stage_mask = off;   off = align_up(off + B * L, A);
+    w.stage_logits = off; off = align_up(off + B * L * 2 * sizeof(float), A);
+    w.slots = ((int64_t)kDecMaxCtas + (int64_t)B * dec_head_groups(c.n_kv_heads)) * kDecWarps;
+    w.part_o = off;       off = align_up(off + (size_t)w.slots * G * kHeadDim * sizeof(float), A);
+    w.part_ml = off;      off = align_up(off + (size_t)w.slots * G * 2 * sizeof(float), A);
+    w.host_q = off;       off = align_up(off + B * c.n_q_heads * kRowBytes, A);
+    w.host_k = off;       off = align_up(off + B * c.n_kv_heads * kRowBytes, A);
+    w.host_v = off;       off = align_up(off + B * c.n_kv_heads * kRowBytes, A);
+    w.host_o = off;       off = align_up(off + B * c.n_q_heads * kRowBytes, A);
+    w.total = off;
+    return w;
+}
+
+static bool aligned16(const void *p) { return (((uintptr_t)p) & 15u) == 0; }
+
+// true if p is device-accessible global memory (device or managed allocation)
+static bool is_device_ptr(const void *p)
+{
+    cudaPointerAttributes a;
+    cudaError_t e = cudaPointerGetAttributes(&a, p);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return a.type == cudaMemoryTypeDevice || a.type == cudaMemoryTypeManaged;
+}
+
+static int need_plan(flux_plan *p, bool need_ws)
+{
+    if (!p) return fail(FLUX_E_INVALID_ARG, "plan is NULL");
+    if (need_ws && !p->ws) return fail(FLUX_E_WORKSPACE, "no workspace set on the plan");
+    return FLUX_OK;
+}
+
+static int need_mask(flux_plan *p, int layer)
+{
+    if (layer < 0 || layer >= p->cfg.n_layers)
+        return fail(FLUX_E_INVALID_ARG, "layer %d outside [0, %d)", layer, p->cfg.n_layers);
+    if (!p->d_mask)
+        return fail(FLUX_E_INVALID_ARG, "flux_router_apply has not been called on this plan");
+    return FLUX_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// small kernels
+// ---------------------------------------------------------------------------------------------
+
+// Hard routing (Sec. 3.1): mask = (pi_FA >= pi_SA), or a validated copy of a given mask.
+__global__ void router_kernel(const float *__restrict__ logits, const uint8_t *__restrict__ mask_in,
+                              uint8_t *__restrict__ mask_out, int n, uint32_t *status)
+{
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    if (mask_in) {
+        uint8_t m = mask_in[i];
+        if (m > 1) {
+            atomicOr(status, FLUX_STATUS_BAD_MASK);
+            m = 1;  // an unreadable decision falls back to the dense mode
+        }
+        mask_out[i] = m;
+    } else {
+        float fa = logits[2 * i], sa = logits[2 * i + 1];
+        if (isnan(fa) || isnan(sa)) {
+            atomicOr(status, FLUX_STATUS_NAN_LOGIT);
+            mask_out[i] = 1;
+        } else {
+            mask_out[i] = (fa >= sa) ? 1 : 0;
+        }
+    }
+}
+
+// Row of the cache that holds position `pos`.
+__device__ __forceinline__ int64_t cache_row(int pos, bool compact_sa, int S, int W)
+{
+    if (!compact_sa || pos < S) return pos;
+    return (int64_t)S + (pos - S) % W;
+}
+
+// One token per request: 16 bytes per thread, K row then V row.
+__global__ void kv_append_kernel(const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
+                                 void *const *__restrict__ k_caches, void *const *__restrict__ v_caches,
+                                 const int32_t *__restrict__ pos, const uint8_t *__restrict__ mask,
+                                 int L, int layer, int row_u4, int S, int W, int layout,
+                                 int max_context, uint32_t *status)
+{
+    const int b = blockIdx.x;
+    const int p = pos[b];
+    if (p < 0) return;
+    if (p >= max_context) {
+        if (threadIdx.x == 0) atomicOr(status, FLUX_STATUS_BAD_LENGTH);
+        return;
+    }
+    const bool compact = (layout == FLUX_KV_COMPACT_SA) && (mask[b * L + layer] == 0);
+    const int64_t row = cache_row(p, compact, S, W);
+    uint4 *kd = (uint4 *)k_caches[b] + row * row_u4;
+    uint4 *vd = (uint4 *)v_caches[b] + row * row_u4;
+    for (int i = threadIdx.x; i < row_u4; i += blockDim.x) {
+        kd[i] = k_new[(int64_t)b * row_u4 + i];
+        vd[i] = v_new[(int64_t)b * row_u4 + i];
+    }
+}
+
+// Prefill -> cache hand-off: copy the rows decode will need (see flux_kv_retain).
+__global__ void kv_retain_kernel(const uint4 *__restrict__ k_src, const uint4 *__restrict__ v_src,
+                                 uint4 *__restrict__ k_dst, uint4 *__restrict__ v_dst, int n,
+                                 const uint8_t *__restrict__ mask, int L, int layer, int req,
+                                 int row_u4, int S, int W, int layout, int copy_identity)
+{
+    const bool compact = (layout == FLUX_KV_COMPACT_SA) && (mask[req * L + layer] == 0);
+    if (!compact && !copy_identity) return;  // source already is the cache
+    // kept rows: [0, a1) and [b0, n); for a full copy a1 = n and the second range is empty
+    const int a1 = compact ? min(S, n) : n;
+    const int b0 = compact ? min(n, max(S, n - W)) : n;
+    const int n_rows = a1 + (n - b0);
+    for (int r = blockIdx.x; r < n_rows; r += gridDim.x) {
+        const int p = r < a1 ? r : b0 + (r - a1);
+        const int64_t row = cache_row(p, compact, S, W);
+        for (int i = threadIdx.x; i < row_u4; i += blockDim.x) {
+            k_dst[row * row_u4 + i] = k_src[(int64_t)p * row_u4 + i];
+            v_dst[row * row_u4 + i] = v_src[(int64_t)p * row_u4 + i];
+        }
+    }
+}
+
+int launch_router(flux_plan *p, const float *d_logits, const uint8_t *d_mask_in, int B,
+                  uint8_t *d_mask_out, cudaStream_t st)
+{
+    const int n = B * p->cfg.n_layers;
+    uint32_t *status = (uint32_t *)((char *)p->ws + p->lay.status);
+    router_kernel<<<(n + 127) / 128, 128, 0, st>>>(d_logits, d_mask_in, d_mask_out, n, status);
+    p->launches++;
+    return check_cuda(cudaGetLastError(), "router kernel launch");
+}
+
+int launch_kv_append(flux_plan *p, int layer, int B, const void *k_new, const void *v_new,
+                     void *const *k_caches, void *const *v_caches, const int32_t *pos,
+                     cudaStream_t st)
+{
+    const flux_config &c = p->cfg;
+    const int row_u4 = c.n_kv_heads * kRowBytes / 16;
+    uint32_t *status = (uint32_t *)((char *)p->ws + p->lay.status);
+    kv_append_kernel<<<B, 128, 0, st>>>((const uint4 *)k_new, (const uint4 *)v_new, k_caches,
+                                        v_caches, pos, p->d_mask, c.n_layers, layer, row_u4,
+                                        c.sink, c.window, c.kv_layout, c.max_context, status);
+    p->launches++;
+    return check_cuda(cudaGetLastError(), "kv_append kernel launch");
+}
+
+int launch_kv_retain(flux_plan *p, int layer, int req, const void *k_src, const void *v_src,
+                     int n, void *k_cache, void *v_cache, cudaStream_t st)
+{
+    const flux_config &c = p->cfg;
+    const int row_u4 = c.n_kv_heads * kRowBytes / 16;
+    const int copy_identity = (k_src != k_cache || v_src != v_cache) ? 1 : 0;
+    int grid = n < 1 ? 1 : (n > p->dev.n_sms * 8 ? p->dev.n_sms * 8 : n);
+    kv_retain_kernel<<<grid, 128, 0, st>>>((const uint4 *)k_src, (const uint4 *)v_src,
+                                           (uint4 *)k_cache, (uint4 *)v_cache, n, p->d_mask,
+                                           c.n_layers, layer, req, row_u4, c.sink, c.window,
+                                           c.kv_layout, copy_identity);
+    p->launches++;
+    return check_cuda(cudaGetLastError(), "kv_retain kernel launch");
+}
+
+}  // namespace flux
+
+using namespace flux;
+
+// ---------------------------------------------------------------------------------------------
+// C ABI
+// ---------------------------------------------------------------------------------------------
+
+extern "C" {
+
+const char *flux_last_error(void) { return g_err; }
+const char *flux_version(void) { return "0.1"; }
+
+int flux_workspace_size(const flux_config *cfg, size_t *bytes_out)
+{
+    int rc = validate_config(cfg);
+    if (rc) return rc;
+    if (!bytes_out) return fail(FLUX_E_INVALID_ARG, "bytes_out is NULL");
+    *bytes_out = workspace_layout(*cfg).total;
+    return FLUX_OK;
+}
+
+int flux_plan_create(const flux_config *cfg, flux_plan **plan)
+{
+    if (plan) *plan = nullptr;
+    int rc = validate_config(cfg);
+    if (rc) return rc;
+    if (!plan) return fail(FLUX_E_INVALID_ARG, "plan out-pointer is NULL");
+    int dev = 0;
+    rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
+    if (rc) return rc;
+    flux_plan *p = new (std::nothrow) flux_plan();
+    if (!p) return fail(FLUX_E_INVALID_ARG, "out of host memory");
+    p->cfg = *cfg;
+    p->G = cfg->n_q_heads / cfg->n_kv_heads;
+    p->scale = cfg->softmax_scale > 0.0f ? cfg->softmax_scale : 1.0f / sqrtf((float)cfg->head_dim);
+    p->scale_log2 = p->scale * 1.4426950408889634f;
+    p->ws = nullptr;
+    p->ws_bytes = 0;
+    p->lay = workspace_layout(*cfg);
+    p->d_mask = nullptr;
+    p->mask_B = 0;
+    p->launches = 0;
+    p->debug_records = 0;
+    cudaError_t e = cudaDeviceGetAttribute(&p->dev.n_sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess)
+        e = cudaDeviceGetAttribute(&p->dev.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e == cudaSuccess)
+        e = cudaDeviceGetAttribute(&p->dev.cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) {
+        delete p;
+        return check_cuda(e, "cudaDeviceGetAttribute");
+    }
+    if (p->dev.cc_major != 10) {
+        int cc = p->dev.cc_major;
+        delete p;
+        return fail(FLUX_E_CUDA, "this library is built for sm_100a only (device is sm_%d0)", cc);
+    }
+    p->dec_ctas = p->dev.n_sms < kDecMaxCtas ? p->dev.n_sms : kDecMaxCtas;
+    rc = decode_setup(p);
+    if (!rc) rc = prefill_setup(p);
+    if (rc) {
+        delete p;
+        return rc;
+    }
+    *plan = p;
+    return FLUX_OK;
+}
+
+int flux_plan_destroy(flux_plan *plan)
+{
+    delete plan;
+    return FLUX_OK;
+}
+
+int flux_plan_set_workspace(flux_plan *plan, void *workspace, size_t bytes)
+{
+    int rc = need_plan(plan, false);
+    if (rc) return rc;
+    if (!workspace || (((uintptr_t)workspace) & 255u))
+        return fail(FLUX_E_INVALID_ARG, "workspace must be a 256-byte aligned device pointer");
+    if (bytes < plan->lay.total)
+        return fail(FLUX_E_WORKSPACE, "workspace of %zu bytes is smaller than the %zu needed", bytes,
+                    plan->lay.total);
+    plan->ws = workspace;
+    plan->ws_bytes = bytes;
+    return FLUX_OK;
+}
+
+int flux_router_apply(flux_plan *plan, const float *logits, const uint8_t *mask_or_null, int32_t B,
+                      uint8_t *mask_out, void *stream)
+{
+    int rc = need_plan(plan, true);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const flux_config &c = plan->cfg;
+    if (B < 1 || B > c.max_batch) return fail(FLUX_E_CAPACITY, "B=%d outside [1, %d]", B, c.max_batch);
+    if (!mask_out) return fail(FLUX_E_INVALID_ARG, "mask_out is NULL");
+    if (!logits && !mask_or_null) return fail(FLUX_E_INVALID_ARG, "neither logits nor a mask given");
+    const size_t n = (size_t)B * c.n_layers;
+    const float *d_logits = nullptr;
+    const uint8_t *d_mask_in = nullptr;
+    if (mask_or_null) {
+        if (is_device_ptr(mask_or_null)) {
+            d_mask_in = mask_or_null;
+        } else {
+            for (size_t i = 0; i < n; ++i)
+                if (mask_or_null[i] > 1)
+                    return fail(FLUX_E_INVALID_ARG, "mask byte %zu is %d, not 0 or 1", i,
+                                (int)mask_or_null[i]);
+            uint8_t *stg = (uint8_t *)plan->ws + plan->lay.stage_mask;
+            rc = check_cuda(cudaMemcpyAsync(stg, mask_or_null, n, cudaMemcpyHostToDevice, st),
+                            "mask upload");
+            if (rc) return rc;
+            d_mask_in = stg;
+        }
+    } else {
+        if (is_device_ptr(logits)) {
+            if (!aligned16(logits)) return fail(FLUX_E_INVALID_ARG, "logits not 16-byte aligned");
+            d_logits = logits;
+        } else {
+            for (size_t i = 0; i < 2 * n; ++i)
+                if (isnan(logits[i])) return fail(FLUX_E_INVALID_ARG, "routing logit %zu is NaN", i);
+            float *stg = (float *)((char *)plan->ws + plan->lay.stage_logits);
+            rc = check_cuda(cudaMemcpyAsync(stg, logits, 2 * n * sizeof(float),
+                                            cudaMemcpyHostToDevice, st), "logits upload");
+            if (rc) return rc;
+            d_logits = stg;
+        }
+    }
+    rc = launch_router(plan, d_logits, d_mask_in, B, mask_out, st);
+    if (rc) return rc;
+    plan->d_mask = mask_out;
+    plan->mask_B = B;
+    return FLUX_OK;
+}
+
+int flux_attn_prefill(flux_plan *plan, int32_t layer, int32_t req, const void *q, const void *k,
+                      const void *v, int32_t q_start, int32_t Nq, void *out, void *stream)
+{
+    int rc = need_plan(plan, true);
+    if (rc) return rc;
+    rc = need_mask(plan, layer);
+    if (rc) return rc;
+    if (req < 0 || req >= plan->mask_B)
+        return fail(FLUX_E_INVALID_ARG, "request %d outside the routed batch of %d", req, plan->mask_B);
+    if (Nq < 0 || q_start < 0) return fail(FLUX_E_INVALID_ARG, "negative q_start or Nq");
+    if ((int64_t)q_start + Nq > plan->cfg.max_context)
+        return fail(FLUX_E_CAPACITY, "q_start + Nq = %lld exceeds max_context %d",
+                    (long long)q_start + Nq, plan->cfg.max_context);
+    if (Nq == 0) return FLUX_OK;
+    if (!q || !k || !v || !out) return fail(FLUX_E_INVALID_ARG, "NULL tensor pointer");
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+        return fail(FLUX_E_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    return launch_prefill(plan, layer, req, q, k, v, q_start, Nq, out, (cudaStream_t)stream);
+}
+
+int flux_kv_retain(flux_plan *plan, int32_t layer, int32_t req, const void *k_src, const void *v_src,
+                   int32_t n, void *k_cache, void *v_cache, void *stream)
+{
+    int rc = need_plan(plan, true);
+    if (rc) return rc;
+    rc = need_mask(plan, layer);
+    if (rc) return rc;
+    if (req < 0 || req >= plan->mask_B)
+        return fail(FLUX_E_INVALID_ARG, "request %d outside the routed batch of %d", req, plan->mask_B);
+    if (n < 0 || n > plan->cfg.max_context)
+        return fail(FLUX_E_CAPACITY, "n=%d outside [0, max_context=%d]", n, plan->cfg.max_context);
+    if (n == 0) return FLUX_OK;
+    if (!k_src || !v_src || !k_cache || !v_cache) return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    if (!aligned16(k_src) || !aligned16(v_src) || !aligned16(k_cache) || !aligned16(v_cache))
+        return fail(FLUX_E_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    return launch_kv_retain(plan, layer, req, k_src, v_src, n, k_cache, v_cache,
+                            (cudaStream_t)stream);
+}
+
+static int check_batch_call(flux_plan *plan, int layer, int B)
+{
+    int rc = need_plan(plan, true);
+    if (rc) return rc;
+    rc = need_mask(plan, layer);
+    if (rc) return rc;
+    if (B < 1 || B > plan->mask_B)
+        return fail(FLUX_E_CAPACITY, "B=%d outside [1, routed batch %d]", B, plan->mask_B);
+    return FLUX_OK;
+}
+
+int flux_kv_append(flux_plan *plan, int32_t layer, int32_t B, const void *k_new, const void *v_new,
+                   void *const *k_caches, void *const *v_caches, const int32_t *pos, void *stream)
+{
+    int rc = check_batch_call(plan, layer, B);
+    if (rc) return rc;
+    if (!k_new || !v_new || !k_caches || !v_caches || !pos)
+        return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    if (!aligned16(k_new) || !aligned16(v_new))
+        return fail(FLUX_E_INVALID_ARG, "k_new / v_new must be 16-byte aligned");
+    return launch_kv_append(plan, layer, B, k_new, v_new, k_caches, v_caches, pos,
+                            (cudaStream_t)stream);
+}
+
+int flux_attn_decode(flux_plan *plan, int32_t layer, int32_t B, const void *q,
+                     const void *const *k_caches, const void *const *v_caches,
+                     const int32_t *ctx_len, void *out, void *stream)
+{
+    int rc = check_batch_call(plan, layer, B);
+    if (rc) return rc;
+    if (!q || !k_caches || !v_caches || !ctx_len || !out)
+        return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    if (!aligned16(q) || !aligned16(out))
+        return fail(FLUX_E_INVALID_ARG, "q / out must be 16-byte aligned");
+    return launch_decode(plan, layer, B, q, k_caches, v_caches, ctx_len, out, (cudaStream_t)stream);
+}
+
+int flux_attn_decode_host(flux_plan *plan, int32_t layer, int32_t B, const void *q_host,
+                          const void *k_new_host, const void *v_new_host, void *const *k_caches,
+                          void *const *v_caches, const int32_t *pos, const int32_t *ctx_len,
+                          void *out_host, void *stream)
+{
+    int rc = check_batch_call(plan, layer, B);
+    if (rc) return rc;
+    if (!q_host || !k_new_host || !v_new_host || !k_caches || !v_caches || !pos || !ctx_len ||
+        !out_host)
+        return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    cudaStream_t st = (cudaStream_t)stream;
+    const flux_config &c = plan->cfg;
+    char *ws = (char *)plan->ws;
+    void *dq = ws + plan->lay.host_q, *dk = ws + plan->lay.host_k, *dv = ws + plan->lay.host_v,
+         *dout = ws + plan->lay.host_o;
+    const size_t qb = (size_t)B * c.n_q_heads * kRowBytes, kb = (size_t)B * c.n_kv_heads * kRowBytes;
+    rc = check_cuda(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, st), "q upload");
+    if (!rc) rc = check_cuda(cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, st), "k upload");
+    if (!rc) rc = check_cuda(cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, st), "v upload");
+    if (!rc) rc = launch_kv_append(plan, layer, B, dk, dv, k_caches, v_caches, pos, st);
+    if (!rc)
+        rc = launch_decode(plan, layer, B, dq, (const void *const *)k_caches,
+                           (const void *const *)v_caches, ctx_len, dout, st);
+    if (!rc) rc = check_cuda(cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, st), "out download");
+    return rc;
+}
+
+int flux_attn_prefill_host(flux_plan *plan, int32_t layer, int32_t req, const void *q_host,
+                           void *q_dev, const void *k, const void *v, int32_t q_start, int32_t Nq,
+                           void *out_dev, void *out_host, void *stream)
+{
+    int rc = need_plan(plan, true);
+    if (rc) return rc;
+    if (Nq < 0) return fail(FLUX_E_INVALID_ARG, "negative Nq");
+    if (Nq == 0) return FLUX_OK;
+    if (!q_host || !q_dev || !out_dev || !out_host) return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t qb = (size_t)Nq * plan->cfg.n_q_heads * kRowBytes;
+    rc = check_cuda(cudaMemcpyAsync(q_dev, q_host, qb, cudaMemcpyHostToDevice, st), "q upload");
+    if (!rc) rc = flux_attn_prefill(plan, layer, req, q_dev, k, v, q_start, Nq, out_dev, stream);
+    if (!rc) rc = check_cuda(cudaMemcpyAsync(out_host, out_dev, qb, cudaMemcpyDeviceToHost, st), "out download");
+    return rc;
+}
+
+int flux_plan_status(flux_plan *plan, uint32_t *status_bits, void *stream)
+{
+    int rc = need_plan(plan, true);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint32_t bits = 0;
+    void *d = (char *)plan->ws + plan->lay.status;
+    rc = check_cuda(cudaMemcpyAsync(&bits, d, sizeof bits, cudaMemcpyDeviceToHost, st), "status read");
+    if (!rc) rc = check_cuda(cudaMemsetAsync(d, 0, sizeof bits, st), "status clear");
+    if (!rc) rc = check_cuda(cudaStreamSynchronize(st), "stream synchronize");
+    if (rc) return rc;
+    if (status_bits) *status_bits = bits;
+    if (bits & FLUX_STATUS_WAIT_EXPIRED)
+        return fail(FLUX_E_DEVICE_TIMEOUT, "a device-side wait expired (status 0x%x)", bits);
+    if (bits) return fail(FLUX_E_DEVICE_FLAG, "device-side input check failed (status 0x%x)", bits);
+    return FLUX_OK;
+}
+
+int flux_debug_dispatch(flux_plan *plan, int32_t *records_out, int32_t max_records,
+                        int32_t *n_records_out, void *stream)
+{
+    int rc = need_plan(plan, true);
+    if (rc) return rc;
+    if (!records_out || !n_records_out || max_records < 0)
+        return fail(FLUX_E_INVALID_ARG, "bad output arguments");
+    cudaStream_t st = (cudaStream_t)stream;
+    int n = plan->debug_records < max_records ? plan->debug_records : max_records;
+    if (n > 0) {
+        rc = check_cuda(cudaMemcpyAsync(records_out, (char *)plan->ws + plan->lay.debug,
+                                        (size_t)n * 8 * sizeof(int32_t), cudaMemcpyDeviceToHost, st),
+                        "dispatch record read");
+        if (rc) return rc;
+    }
+    rc = check_cuda(cudaStreamSynchronize(st), "stream synchronize");
+    if (rc) return rc;
+    *n_records_out = n;
+    return FLUX_OK;
+}
+
+int64_t flux_launch_count(const flux_plan *plan) { return plan ? plan->launches : 0; }
+
+}  // extern "C"

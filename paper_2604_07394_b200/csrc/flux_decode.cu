@@ -1,0 +1,539 @@
+// Split-K flash-decode for a batch with mixed FA / SA layers (sm_100a).
+//
+// One launch serves every request of the batch for one layer.  A request in FA
+// mode streams its whole KV cache (Eq. 1); a request in SA mode streams only the
+// sink rows and the window rows (Eq. 2 with the streaming subset; Appendix C.3:
+// the sparse layer "fetches only the locally required KV").  The kept rows of
+// all requests are laid end to end in units of `slices * kDecTile` tokens and cut
+// into gridDim.x equal spans, so every SM streams the same number of bytes
+// whatever the mix of modes and lengths.  Inside a CTA each warp owns one KV
+// head (and one token slice), so the CTA as a whole reads whole token rows of the
+// token-major cache: contiguous, 16-byte vectorised cp.async traffic, no
+// block-level barrier anywhere.  Each warp keeps a flash-attention state
+// (running max, sum, fp32 accumulator) for the G query heads of its KV head,
+// computes QK^T and PV with bf16 tensor-core MMAs (m16n8k16, rows padded to 16),
+// and writes one partial (O, m, l) per segment it touched; a small combine kernel
+// merges the partials (the split-K identity: sums over disjoint key sets merge by
+// rescaling with exp(m_p - m)).
+#include "flux_internal.h"
+
+namespace flux {
+namespace {
+
+constexpr float kNegBig = -1.0e30f;  // finite stand-in for "no key seen yet"
+
+struct DecArgs {
+    const __nv_bfloat16 *q;
+    const void *const *k_caches;
+    const void *const *v_caches;
+    const int32_t *ctx_len;
+    const uint8_t *mask;
+    int B, L, layer, Hq, Hkv, G, S, W, layout, max_context;
+    float scale_log2;
+    float *part_o;
+    float *part_ml;
+    int32_t *debug;
+    int32_t *sched;
+    uint32_t *status;
+    __nv_bfloat16 *out;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3,
+                                            uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t &r0, uint32_t &r1, uint32_t &r2,
+                                                  uint32_t &r3, uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%0,%1,%2,%3};\n"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// What one request contributes to this layer's launch.
+struct ReqInfo {
+    int n;       // context length after clamping
+    int mode;    // 1 FA, 0 SA
+    int n_eff;   // rows the kernel reads
+    int split;   // virtual rows >= split are shifted by `shift` (window part of a FULL cache)
+    int shift;
+};
+
+__device__ __forceinline__ ReqInfo req_info(int n_raw, int mode_raw, int S, int W, int layout,
+                                            int max_context, uint32_t *status)
+{
+    ReqInfo r;
+    int n = n_raw;
+    if (n > max_context) {
+        atomicOr(status, FLUX_STATUS_BAD_LENGTH);
+        n = max_context;
+    }
+    if (n < 0) n = 0;
+    if (mode_raw > 1) atomicOr(status, FLUX_STATUS_BAD_MASK);
+    r.n = n;
+    r.mode = mode_raw != 0 ? 1 : 0;
+    r.split = 0x7fffffff;
+    r.shift = 0;
+    if (r.mode == 1 || n <= S + W) {
+        r.n_eff = n;  // SA with sink + window >= n keeps every row
+    } else {
+        r.n_eff = S + W;
+        if (layout == FLUX_KV_FULL) {  // rows [0,S) then rows [n-W, n)
+            r.split = S;
+            r.shift = n - W - S;
+        }  // COMPACT_SA: the S + W slots are exactly the kept rows, in slot order
+    }
+    return r;
+}
+
+// position of the unit a warp is loading or consuming
+struct UnitIt {
+    int u;      // global unit index
+    int b;      // request
+    int hg;     // head group
+    int x;      // CTA tile inside the request
+    int tiles;  // CTA tiles of request b
+};
+
+__global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    __shared__ int s_prefix[kMaxBatch + 1];
+    __shared__ int s_neff[kMaxBatch];
+    __shared__ int s_split[kMaxBatch];
+    __shared__ int s_shift[kMaxBatch];
+    __shared__ int s_units[kMaxBatch];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int hpc = a.Hkv < kDecWarps ? a.Hkv : kDecWarps;
+    const int slices = kDecWarps / hpc;
+    const int n_hg = (a.Hkv + hpc - 1) / hpc;
+    const int cta_tok = slices * kDecTile;
+
+    // ---- schedule: units per request, prefix sum, equal spans -------------------------------
+    for (int b = tid; b < a.B; b += blockDim.x) {
+        ReqInfo r = req_info(a.ctx_len[b], a.mask[b * a.L + a.layer], a.S, a.W, a.layout,
+                             a.max_context, a.status);
+        s_neff[b] = r.n_eff;
+        s_split[b] = r.split;
+        s_shift[b] = r.shift;
+        s_units[b] = (r.n_eff + cta_tok - 1) / cta_tok * n_hg;
+        if (blockIdx.x == 0) {
+            int32_t *d = a.debug + b * 8;
+            d[0] = r.mode; d[1] = a.layer; d[2] = b; d[3] = r.n;
+            d[4] = 0;
+            d[5] = (r.split < r.n_eff) ? r.split : r.n_eff;
+            d[6] = (r.split < r.n_eff) ? r.split + r.shift : 0;
+            d[7] = (r.split < r.n_eff) ? r.n_eff + r.shift : 0;
+        }
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const int chunk = (a.B + 31) / 32;
+        const int lo = lane * chunk, hi = min(a.B, lo + chunk);
+        int sum = 0;
+        for (int b = lo; b < hi; ++b) sum += s_units[b];
+        int incl = sum;
+        for (int d = 1; d < 32; d <<= 1) {
+            int t = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += t;
+        }
+        int run = incl - sum;
+        for (int b = lo; b < hi; ++b) {
+            s_prefix[b] = run;
+            run += s_units[b];
+        }
+        if (lane == 31) s_prefix[a.B] = incl;
+    }
+    __syncthreads();
+    const int total = s_prefix[a.B];
+    const int span = total > 0 ? (total + gridDim.x - 1) / gridDim.x : 1;
+    if (blockIdx.x == 0) {
+        for (int b = tid; b <= a.B; b += blockDim.x) a.sched[b] = s_prefix[b];
+        if (tid == 0) a.sched[a.B + 1] = span;
+    }
+    const int u_begin = blockIdx.x * span;
+    const int u_end = min(total, u_begin + span);
+    if (u_begin >= u_end) return;
+    const int slice = warp / hpc, hw = warp % hpc;
+    if (slice >= slices) return;
+
+    // ---- iterators ------------------------------------------------------------------------------
+    UnitIt first;
+    {
+        int lo = 0, hi = a.B - 1;  // last b with prefix[b] <= u_begin and units > 0
+        while (lo < hi) {
+            int mid = (lo + hi + 1) >> 1;
+            if (s_prefix[mid] <= u_begin) lo = mid; else hi = mid - 1;
+        }
+        while (s_units[lo] == 0 && lo + 1 < a.B) ++lo;  // cannot trigger: u_begin < total
+        first.u = u_begin;
+        first.b = lo;
+        first.tiles = s_units[lo] / n_hg;
+        const int off = u_begin - s_prefix[lo];
+        first.hg = off / first.tiles;
+        first.x = off % first.tiles;
+    }
+    auto advance = [&](UnitIt &it) {
+        ++it.u;
+        if (it.u >= u_end) return;
+        if (++it.x == it.tiles) {
+            it.x = 0;
+            if (++it.hg == n_hg) {
+                it.hg = 0;
+                do { ++it.b; } while (s_units[it.b] == 0);
+                it.tiles = s_units[it.b] / n_hg;
+            }
+        }
+    };
+
+    unsigned char *my_smem = smem + (size_t)warp * kDecStages * kDecStageBytes;
+    const uint32_t my_smem_u32 = smem_u32(my_smem);
+
+    // loader state
+    UnitIt lit = first;
+    int l_b = -1;
+    const unsigned char *l_k = nullptr, *l_v = nullptr;
+    const int lc = lane & 15, lr0 = lane >> 4;
+    auto issue = [&](int stage) {
+        const int head = lit.hg * hpc + hw;
+        if (head < a.Hkv) {
+            if (lit.b != l_b) {
+                l_b = lit.b;
+                l_k = (const unsigned char *)a.k_caches[l_b];
+                l_v = (const unsigned char *)a.v_caches[l_b];
+            }
+            const int n_eff = s_neff[l_b], split = s_split[l_b], shift = s_shift[l_b];
+            const int v0 = (lit.x * slices + slice) * kDecTile;
+            const uint32_t sbase = my_smem_u32 + stage * kDecStageBytes;
+#pragma unroll
+            for (int i = 0; i < kDecTile / 2; ++i) {
+                const int r = lr0 + 2 * i;
+                const int v = v0 + r;
+                const bool valid = v < n_eff;
+                const int pos = valid ? (v >= split ? v + shift : v) : 0;
+                const size_t off = ((size_t)pos * a.Hkv + head) * kRowBytes + lc * 16;
+                const uint32_t dst = sbase + r * kRowBytes + ((lc ^ (r & 7)) << 4);
+                cp_async16(dst, l_k + off, valid ? 16 : 0);
+                cp_async16(dst + kDecTile * kRowBytes, l_v + off, valid ? 16 : 0);
+            }
+        }
+        cp_async_commit();
+    };
+
+    const int n_units = u_end - u_begin;
+#pragma unroll
+    for (int s = 0; s < kDecStages - 1; ++s) {
+        if (s < n_units) {
+            issue(s);
+            advance(lit);
+        } else {
+            cp_async_commit();
+        }
+    }
+
+    // consumer state
+    UnitIt cit = first;
+    int cur_seg = -1;
+    bool cur_active = false;
+    float o[16][4];
+    float m_r[2], l_r[2];
+    uint32_t qf[8][4];
+    const int g = lane >> 2, t4 = lane & 3;
+
+    auto flush = [&]() {
+        if (cur_seg < 0 || !cur_active) return;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            l_r[i] += __shfl_xor_sync(0xffffffffu, l_r[i], 1);
+            l_r[i] += __shfl_xor_sync(0xffffffffu, l_r[i], 2);
+        }
+        const size_t slot = ((size_t)blockIdx.x + cur_seg) * kDecWarps + warp;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int row = g + 8 * i;
+            if (row < a.G) {
+                float *po = a.part_o + (slot * a.G + row) * kHeadDim;
+#pragma unroll
+                for (int nt = 0; nt < 16; ++nt)
+                    *reinterpret_cast<float2 *>(po + nt * 8 + 2 * t4) =
+                        make_float2(o[nt][2 * i], o[nt][2 * i + 1]);
+                if (t4 == 0) {
+                    float *pm = a.part_ml + (slot * a.G + row) * 2;
+                    pm[0] = m_r[i];
+                    pm[1] = l_r[i];
+                }
+            }
+        }
+    };
+
+    for (int t = 0; t < n_units; ++t) {
+        cp_async_wait<kDecStages - 2>();
+        __syncwarp();
+        if (t + kDecStages - 1 < n_units) {
+            issue((t + kDecStages - 1) % kDecStages);
+            advance(lit);
+        } else {
+            cp_async_commit();
+        }
+
+        const int seg = cit.b * n_hg + cit.hg;
+        if (seg != cur_seg) {
+            flush();
+            cur_seg = seg;
+            const int head = cit.hg * hpc + hw;
+            cur_active = head < a.Hkv;
+            if (cur_active) {
+#pragma unroll
+                for (int nt = 0; nt < 16; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) o[nt][e] = 0.f;
+                m_r[0] = m_r[1] = kNegBig;
+                l_r[0] = l_r[1] = 0.f;
+                const __nv_bfloat16 *qb = a.q + ((size_t)cit.b * a.Hq + (size_t)head * a.G) * kHeadDim;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int row = g + 8 * (e & 1);
+                        const int col = kk * 16 + 2 * t4 + 8 * (e >> 1);
+                        qf[kk][e] = row < a.G
+                                        ? *reinterpret_cast<const uint32_t *>(qb + (size_t)row * kHeadDim + col)
+                                        : 0u;
+                    }
+                }
+            }
+        }
+
+        if (cur_active) {
+            const int stage = t % kDecStages;
+            const uint32_t kb = my_smem_u32 + stage * kDecStageBytes;
+            const uint32_t vb = kb + kDecTile * kRowBytes;
+            const int v0 = (cit.x * slices + slice) * kDecTile;
+            const int n_valid = s_neff[cit.b] - v0;  // may be <= 0 for a trailing empty slice
+
+            // S = Q K^T for 16 keys
+            float s[2][4];
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) s[j][e] = 0.f;
+            {
+                const int mi = lane >> 3, rr = lane & 7;
+                const int key = (mi >> 1) * 8 + rr;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const int chunk = kk * 2 + (mi & 1);
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4(b0, b1, b2, b3, kb + key * kRowBytes + ((chunk ^ rr) << 4));
+                    mma_bf16(s[0], qf[kk], b0, b1);
+                    mma_bf16(s[1], qf[kk], b2, b3);
+                }
+            }
+            // scale into the log2 domain, mask the ragged tail
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int key = j * 8 + 2 * t4 + (e & 1);
+                    s[j][e] = key < n_valid ? s[j][e] * a.scale_log2 : -INFINITY;
+                }
+            // online softmax for rows g and g + 8
+            float alpha[2];
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                float mx = fmaxf(fmaxf(s[0][2 * i], s[0][2 * i + 1]), fmaxf(s[1][2 * i], s[1][2 * i + 1]));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float m_new = fmaxf(m_r[i], mx);
+                alpha[i] = fast_exp2(m_r[i] - m_new);
+                m_r[i] = m_new;
+                float rs = 0.f;
+#pragma unroll
+                for (int j = 0; j < 2; ++j)
+#pragma unroll
+                    for (int e = 0; e < 2; ++e) {
+                        const float p = fast_exp2(s[j][2 * i + e] - m_new);
+                        s[j][2 * i + e] = p;
+                        rs += p;
+                    }
+                l_r[i] = l_r[i] * alpha[i] + rs;
+            }
+            uint32_t pa[4];
+            pa[0] = pack_bf16(s[0][0], s[0][1]);
+            pa[1] = pack_bf16(s[0][2], s[0][3]);
+            pa[2] = pack_bf16(s[1][0], s[1][1]);
+            pa[3] = pack_bf16(s[1][2], s[1][3]);
+            // O = alpha * O + P V
+            {
+                const int mi = lane >> 3, rr = lane & 7;
+                const int key = (mi & 1) * 8 + rr;
+#pragma unroll
+                for (int dt = 0; dt < 8; ++dt) {
+                    const int chunk = dt * 2 + (mi >> 1);
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4_trans(b0, b1, b2, b3, vb + key * kRowBytes + ((chunk ^ rr) << 4));
+#pragma unroll
+                    for (int h2 = 0; h2 < 2; ++h2) {
+                        float(&acc)[4] = o[2 * dt + h2];
+                        acc[0] *= alpha[0];
+                        acc[1] *= alpha[0];
+                        acc[2] *= alpha[1];
+                        acc[3] *= alpha[1];
+                    }
+                    mma_bf16(o[2 * dt], pa, b0, b1);
+                    mma_bf16(o[2 * dt + 1], pa, b2, b3);
+                }
+            }
+        }
+        advance(cit);
+    }
+    flush();
+    cp_async_wait<0>();
+}
+
+// Merge the partials of one (request, query head) and write the bf16 output row.
+__global__ void __launch_bounds__(128) decode_combine_kernel(DecArgs a)
+{
+    __shared__ float s_o[4][kHeadDim];
+    __shared__ float s_m[4], s_l[4];
+    const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int hpc = a.Hkv < kDecWarps ? a.Hkv : kDecWarps;
+    const int slices = kDecWarps / hpc;
+    const int n_hg = (a.Hkv + hpc - 1) / hpc;
+    __nv_bfloat16 *dst = a.out + ((size_t)b * a.Hq + h) * kHeadDim;
+
+    const int ustart = a.sched[b], uend = a.sched[b + 1], span = a.sched[a.B + 1];
+    const int units = uend - ustart;
+    if (units == 0) {  // inactive request
+        dst[threadIdx.x] = __float2bfloat16(0.f);
+        return;
+    }
+    const int tiles = units / n_hg;
+    const int kvh = h / a.G, r = h % a.G;
+    const int hg = kvh / hpc, hw = kvh % hpc;
+    const int us = ustart + hg * tiles, ue = us + tiles;
+    const int c_first = us / span, c_last = (ue - 1) / span;
+    const int seg = b * n_hg + hg;
+    const int n_part = (c_last - c_first + 1) * slices;
+
+    float m = kNegBig, l = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int p = warp; p < n_part; p += 4) {
+        const int c = c_first + p / slices, s = p % slices;
+        const size_t slot = ((size_t)c + seg) * kDecWarps + (hw + hpc * s);
+        const float *pm = a.part_ml + (slot * a.G + r) * 2;
+        const float mp = pm[0], lp = pm[1];
+        const float4 op = *reinterpret_cast<const float4 *>(a.part_o + (slot * a.G + r) * kHeadDim + lane * 4);
+        const float m_new = fmaxf(m, mp);
+        const float so = fast_exp2(m - m_new), sp = fast_exp2(mp - m_new);
+        acc.x = acc.x * so + op.x * sp;
+        acc.y = acc.y * so + op.y * sp;
+        acc.z = acc.z * so + op.z * sp;
+        acc.w = acc.w * so + op.w * sp;
+        l = l * so + lp * sp;
+        m = m_new;
+    }
+    *reinterpret_cast<float4 *>(&s_o[warp][lane * 4]) = acc;
+    if (lane == 0) {
+        s_m[warp] = m;
+        s_l[warp] = l;
+    }
+    __syncthreads();
+    const int d = threadIdx.x;
+    float mm = fmaxf(fmaxf(s_m[0], s_m[1]), fmaxf(s_m[2], s_m[3]));
+    float num = 0.f, den = 0.f;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        const float sc = fast_exp2(s_m[w] - mm);
+        num += s_o[w][d] * sc;
+        den += s_l[w] * sc;
+    }
+    dst[d] = __float2bfloat16(den > 0.f ? num / den : 0.f);
+}
+
+constexpr int kDecSmemBytes = kDecWarps * kDecStages * kDecStageBytes;
+
+}  // namespace
+
+int decode_setup(flux_plan *p)
+{
+    if (p->dev.smem_optin < kDecSmemBytes)
+        return fail(FLUX_E_CUDA, "device offers %d bytes of shared memory per block, decode needs %d",
+                    p->dev.smem_optin, kDecSmemBytes);
+    return check_cuda(cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           kDecSmemBytes),
+                      "cudaFuncSetAttribute(decode_kernel)");
+}
+
+int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *const *k_caches,
+                  const void *const *v_caches, const int32_t *ctx_len, void *out, cudaStream_t st)
+{
+    const flux_config &c = p->cfg;
+    char *ws = (char *)p->ws;
+    DecArgs a;
+    a.q = (const __nv_bfloat16 *)q;
+    a.k_caches = k_caches;
+    a.v_caches = v_caches;
+    a.ctx_len = ctx_len;
+    a.mask = p->d_mask;
+    a.B = B; a.L = c.n_layers; a.layer = layer; a.Hq = c.n_q_heads; a.Hkv = c.n_kv_heads;
+    a.G = p->G; a.S = c.sink; a.W = c.window; a.layout = c.kv_layout; a.max_context = c.max_context;
+    a.scale_log2 = p->scale_log2;
+    a.part_o = (float *)(ws + p->lay.part_o);
+    a.part_ml = (float *)(ws + p->lay.part_ml);
+    a.debug = (int32_t *)(ws + p->lay.debug);
+    a.sched = (int32_t *)(ws + p->lay.sched);
+    a.status = (uint32_t *)(ws + p->lay.status);
+    a.out = (__nv_bfloat16 *)out;
+    decode_kernel<<<p->dec_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
+    p->launches++;
+    int rc = check_cuda(cudaGetLastError(), "decode kernel launch");
+    if (rc) return rc;
+    decode_combine_kernel<<<B * c.n_q_heads, 128, 0, st>>>(a);
+    p->launches++;
+    p->debug_records = B;
+    return check_cuda(cudaGetLastError(), "decode combine kernel launch");
+}
+
+}  // namespace flux

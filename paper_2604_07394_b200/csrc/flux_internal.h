@@ -1,0 +1,98 @@
+// Internal declarations shared by the translation units of libflux_attn.so.
+// Nothing here is part of the public ABI (see include/flux_attn.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "flux_attn.h"
+
+namespace flux {
+
+constexpr int kHeadDim = 128;
+constexpr int kRowBytes = kHeadDim * 2;  // one head of one token, bf16
+
+// ---- decode kernel geometry -------------------------------------------------
+constexpr int kDecWarps = 8;        // warps per CTA, each an independent streaming pipeline
+constexpr int kDecTile = 16;        // tokens per pipeline stage of one warp
+constexpr int kDecStages = 3;       // cp.async stages per warp
+constexpr int kDecStageBytes = kDecTile * kRowBytes * 2;  // K tile + V tile
+constexpr int kDecMaxCtas = 512;    // upper bound used to size the workspace
+constexpr int kMaxBatch = 1024;     // prefix tables live in shared memory
+
+// ---- workspace layout (byte offsets from the workspace base) ----------------
+struct WorkspaceLayout {
+    size_t status;       // uint32 status word (+ padding)
+    size_t debug;        // int32 [max_batch][8] dispatch records
+    size_t sched;        // int32 [max_batch + 4] decode schedule table (prefix, span)
+    size_t stage_mask;   // uint8 [max_batch][L]
+    size_t stage_logits; // fp32  [max_batch][L][2]
+    size_t part_o;       // fp32  [slots][G][D]
+    size_t part_ml;      // fp32  [slots][G][2]
+    size_t host_q;       // bf16  [max_batch][Hq][D]   staging for *_host calls
+    size_t host_k;       // bf16  [max_batch][Hkv][D]
+    size_t host_v;       // bf16  [max_batch][Hkv][D]
+    size_t host_o;       // bf16  [max_batch][Hq][D]
+    size_t total;
+    int64_t slots;
+};
+
+WorkspaceLayout workspace_layout(const flux_config &cfg);
+
+// heads of one KV-head group a decode CTA serves at once, and token slices per CTA tile
+inline int dec_heads_per_cta(int Hkv) { return Hkv < kDecWarps ? Hkv : kDecWarps; }
+inline int dec_slices(int Hkv) { return kDecWarps / dec_heads_per_cta(Hkv); }
+inline int dec_head_groups(int Hkv)
+{
+    int hpc = dec_heads_per_cta(Hkv);
+    return (Hkv + hpc - 1) / hpc;
+}
+
+struct Dev {
+    int n_sms;
+    int smem_optin;
+    int cc_major;
+};
+
+}  // namespace flux
+
+struct flux_plan {
+    flux_config cfg;
+    flux::Dev dev;
+    int G;
+    float scale;        // softmax scale
+    float scale_log2;   // scale * log2(e)
+    void *ws;
+    size_t ws_bytes;
+    flux::WorkspaceLayout lay;
+    const uint8_t *d_mask;  // cached routing decision [mask_B][L], device
+    int32_t mask_B;
+    int64_t launches;
+    int32_t debug_records;  // records the latest call wrote
+    int dec_ctas;
+};
+
+namespace flux {
+
+// error bookkeeping (flux_api.cu)
+int fail(int code, const char *fmt, ...);
+int check_cuda(cudaError_t e, const char *what);
+
+// kernel launchers; each returns FLUX_OK or a negative code and bumps plan->launches
+int launch_router(flux_plan *p, const float *d_logits, const uint8_t *d_mask_in, int B,
+                  uint8_t *d_mask_out, cudaStream_t st);
+int launch_kv_append(flux_plan *p, int layer, int B, const void *k_new, const void *v_new,
+                     void *const *k_caches, void *const *v_caches, const int32_t *pos,
+                     cudaStream_t st);
+int launch_kv_retain(flux_plan *p, int layer, int req, const void *k_src, const void *v_src,
+                     int n, void *k_cache, void *v_cache, cudaStream_t st);
+int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *const *k_caches,
+                  const void *const *v_caches, const int32_t *ctx_len, void *out,
+                  cudaStream_t st);
+int launch_prefill(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v,
+                   int q_start, int Nq, void *out, cudaStream_t st);
+int decode_setup(flux_plan *p);   // one-time attribute setting for the decode kernel
+int prefill_setup(flux_plan *p);
+
+}  // namespace flux

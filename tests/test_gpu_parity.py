@@ -1,0 +1,284 @@
+"""GPU parity: the CUDA path (through the C ABI) against the fp64 oracle, element by element,
+on the same seeded inputs.  Small shapes are swept in full; they span several tiles and ragged
+tails.  Dispatch (mask bytes) and the KV rows each layer reads are compared bit-exactly."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_07394_b200 import synth
+from tests._util import bits, compact_rows_to_positions, compare, expand_ranges, logical_view
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module")
+def flux():
+    from paper_2604_07394_b200 import build, flux as f
+    build.build()
+    f.load()
+    return f
+
+
+def _scale(D=128):
+    return 1.0 / np.sqrt(D)
+
+
+def _plan(flux, L, Hq, Hkv, S, W, B, max_ctx, layout=0):
+    cfg = flux.make_config(L, Hq, Hkv, S, W, B, max_ctx, kv_layout=layout)
+    return flux.Plan(cfg, DEV)
+
+
+# ---- configuration 1 in full: prefill ---------------------------------------------------------
+
+def test_cfg1_prefill_every_row(flux):
+    w = synth.WORKLOADS["cfg1"]
+    mask = synth.layer_masks(w)
+    logits = synth.masks_to_logits(mask, w.seed)
+    plan = _plan(flux, w.n_layers, w.n_q_heads, w.n_kv_heads, w.sink, w.window, 1, 2048)
+    mask_dev = plan.flux_router_apply(logits=torch.from_numpy(logits).to(DEV))
+    assert np.array_equal(mask_dev.cpu().numpy(), oracle.route(logits))
+    assert mask.tolist() == [[1, 0, 1, 0]]
+    N = w.prompt_len
+    for layer in range(w.n_layers):
+        q = synth.normal_bf16((N, w.n_q_heads, 128), w.seed, synth.stream_id("q", layer), DEV)
+        k = synth.normal_bf16((N, w.n_kv_heads, 128), w.seed, synth.stream_id("k", layer), DEV)
+        v = synth.normal_bf16((N, w.n_kv_heads, 128), w.seed, synth.stream_id("v", layer), DEV)
+        out = plan.flux_attn_prefill(layer, 0, q, k, v, 0)
+        rec = plan.flux_debug_dispatch(1)
+        ref = oracle.prefill(int(mask[0, layer]), bits(q), bits(k), bits(v), 0, w.sink, w.window, _scale())
+        compare(out, ref, "cfg1 prefill layer %d" % layer)
+        assert rec[0, 0] == mask[0, layer] and rec[0, 1] == layer and rec[0, 3] == N
+        assert expand_ranges(rec[0]) == oracle.kept(int(mask[0, layer]), N - 1, w.sink, w.window).tolist()
+    assert plan.flux_plan_status() == 0
+
+
+# ---- configuration 1 in full: prefill -> retain -> 16 decode steps, both cache layouts -------
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_cfg1_decode_steps(flux, layout):
+    w = synth.WORKLOADS["cfg1"]
+    L, Hq, Hkv, S, W, N, T = w.n_layers, w.n_q_heads, w.n_kv_heads, w.sink, w.window, w.prompt_len, w.decode_steps
+    mask = synth.layer_masks(w)
+    plan = _plan(flux, L, Hq, Hkv, S, W, 1, N + T, layout)
+    plan.flux_router_apply(mask=mask)          # host mask, staged by the library
+    assert np.array_equal(plan.mask.cpu().numpy(), mask)
+    cap_full = N + T
+    kc, vc, kfull, vfull = [], [], [], []
+    for layer in range(L):
+        k = synth.normal_bf16((N, Hkv, 128), w.seed, synth.stream_id("k", layer), DEV)
+        v = synth.normal_bf16((N, Hkv, 128), w.seed, synth.stream_id("v", layer), DEV)
+        compact = layout == 1 and mask[0, layer] == 0
+        rows = S + W if compact else cap_full
+        kcache = torch.zeros((rows, Hkv, 128), dtype=torch.bfloat16, device=DEV)
+        vcache = torch.zeros_like(kcache)
+        plan.flux_kv_retain(layer, 0, k, v, N, kcache, vcache)
+        kc.append(kcache); vc.append(vcache)
+        kfull.append(torch.cat([k.cpu(), torch.zeros((T, Hkv, 128), dtype=torch.bfloat16)]))
+        vfull.append(torch.cat([v.cpu(), torch.zeros((T, Hkv, 128), dtype=torch.bfloat16)]))
+    ktab = [flux.pointer_table([kc[l]], DEV) for l in range(L)]
+    vtab = [flux.pointer_table([vc[l]], DEV) for l in range(L)]
+    for step in range(T):
+        n = N + step + 1
+        pos = torch.tensor([n - 1], dtype=torch.int32, device=DEV)
+        ctx = torch.tensor([n], dtype=torch.int32, device=DEV)
+        for layer in range(L):
+            mode = int(mask[0, layer])
+            compact = layout == 1 and mode == 0
+            qd = synth.normal_bf16((1, Hq, 128), w.seed, synth.stream_id("qdec", layer, 0, step), DEV)
+            kn = synth.normal_bf16((1, Hkv, 128), w.seed, synth.stream_id("kdec", layer, 0, step), DEV)
+            vn = synth.normal_bf16((1, Hkv, 128), w.seed, synth.stream_id("vdec", layer, 0, step), DEV)
+            plan.flux_kv_append(layer, 1, kn, vn, ktab[layer], vtab[layer], pos)
+            out = plan.flux_attn_decode(layer, 1, qd, ktab[layer], vtab[layer], ctx)
+            rec = plan.flux_debug_dispatch(1)
+            kfull[layer][n - 1] = kn[0].cpu(); vfull[layer][n - 1] = vn[0].cpu()
+            ref = oracle.decode(mode, bits(qd[0]), bits(kfull[layer]), bits(vfull[layer]), n, S, W, _scale())
+            compare(out[0], ref, "cfg1 decode step %d layer %d layout %d" % (step, layer, layout))
+            # dispatch and the set of KV rows read, bit-exact
+            assert rec[0, 0] == mode and rec[0, 3] == n
+            rows = expand_ranges(rec[0])
+            want = oracle.kept(mode, n - 1, S, W).tolist()
+            if compact:
+                assert compact_rows_to_positions(rows, n, S, W) == want
+            else:
+                assert rows == want
+            if step in (0, T - 1):   # the cache itself holds what the oracle says must be retained
+                kv = logical_view(kc[layer], n, S, W, compact)
+                keep = oracle.retained(n, S, W) if mode == 0 else np.arange(n)
+                assert torch.equal(kv[keep], kfull[layer][:n][keep])
+    assert plan.flux_plan_status() == 0
+
+
+# ---- small shapes: tiles, ragged tails, degenerate sink / window, GQA widths ------------------
+
+PREFILL_CASES = [
+    # N, Hq, Hkv, S, W, q_start-chunks
+    (1, 4, 2, 4, 8, None),
+    (63, 4, 2, 4, 8, None),
+    (64, 4, 4, 0, 1, None),
+    (65, 8, 2, 64, 64, None),
+    (130, 7, 1, 3, 70, None),
+    (300, 28, 4, 128, 100, None),
+    (257, 8, 2, 0, 64, None),
+    (400, 8, 8, 70, 129, (0, 100, 164, 400)),
+    (520, 4, 1, 64, 256, (0, 512, 520)),
+]
+
+
+@pytest.mark.parametrize("N,Hq,Hkv,S,W,chunks", PREFILL_CASES)
+def test_prefill_small_shapes(flux, N, Hq, Hkv, S, W, chunks):
+    plan = _plan(flux, 2, Hq, Hkv, S, W, 1, 1024)
+    plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
+    seed = 1000 + N
+    q = synth.normal_bf16((N, Hq, 128), seed, 1, DEV)
+    k = synth.normal_bf16((N, Hkv, 128), seed, 2, DEV)
+    v = synth.normal_bf16((N, Hkv, 128), seed, 3, DEV)
+    for layer, mode in ((0, oracle.FA), (1, oracle.SA)):
+        ref = oracle.prefill(mode, bits(q), bits(k), bits(v), 0, S, W, _scale())
+        if chunks is None:
+            out = plan.flux_attn_prefill(layer, 0, q, k, v, 0)
+        else:
+            out = torch.empty_like(q)
+            for a, b in zip(chunks[:-1], chunks[1:]):
+                out[a:b] = plan.flux_attn_prefill(layer, 0, q[a:b].contiguous(), k, v, a)
+        compare(out, ref, "prefill N=%d mode=%d" % (N, mode))
+        rec = plan.flux_debug_dispatch(1)
+        assert expand_ranges(rec[0]) == oracle.kept(mode, N - 1, S, W).tolist()
+    assert plan.flux_plan_status() == 0
+
+
+DECODE_CASES = [
+    # Hq, Hkv, S, W, context lengths (0 = inactive request), layout
+    (8, 2, 4, 8, [1, 12, 13, 40], 0),
+    (8, 2, 4, 8, [1, 12, 13, 40], 1),
+    (28, 4, 16, 48, [64, 65, 300, 5], 0),
+    (28, 4, 16, 48, [64, 65, 300, 5], 1),
+    (6, 3, 0, 1, [7, 1, 33], 0),
+    (16, 1, 8, 32, [500, 0, 41, 17], 1),
+    (32, 8, 128, 256, [1000, 384, 385, 31], 0),
+    (24, 12, 5, 20, [90, 25, 26], 1),
+    (16, 16, 32, 64, [200, 97], 0),
+]
+
+
+@pytest.mark.parametrize("Hq,Hkv,S,W,lens,layout", DECODE_CASES)
+def test_decode_small_shapes(flux, Hq, Hkv, S, W, lens, layout):
+    B = len(lens)
+    L = 2
+    rng = np.random.default_rng(Hq * 100 + Hkv)
+    mask = rng.integers(0, 2, size=(B, L)).astype(np.uint8)
+    mask[0] = [1, 0]
+    cap = max(lens) + 1
+    plan = _plan(flux, L, Hq, Hkv, S, W, B, cap, layout)
+    plan.flux_router_apply(mask=torch.from_numpy(mask).to(DEV))      # device mask
+    for layer in range(L):
+        kc, vc, klog, vlog = [], [], [], []
+        for b, n in enumerate(lens):
+            compact = layout == 1 and mask[b, layer] == 0
+            k = synth.normal_bf16((max(n, 1), Hkv, 128), 77, synth.stream_id("k", layer, b), DEV)
+            v = synth.normal_bf16((max(n, 1), Hkv, 128), 77, synth.stream_id("v", layer, b), DEV)
+            rows = S + W if compact else cap
+            kcache = torch.full((rows, Hkv, 128), float("nan"), dtype=torch.bfloat16, device=DEV)
+            vcache = torch.full_like(kcache, float("nan"))
+            if n > 1:   # all but the newest token come from "prefill"; the newest is appended below
+                plan.flux_kv_retain(layer, b, k, v, n - 1, kcache, vcache)
+            kc.append(kcache); vc.append(vcache); klog.append(k); vlog.append(v)
+        ktab, vtab = flux.pointer_table(kc, DEV), flux.pointer_table(vc, DEV)
+        pos = torch.tensor([n - 1 for n in lens], dtype=torch.int32, device=DEV)
+        ctx = torch.tensor(lens, dtype=torch.int32, device=DEV)
+        kn = torch.stack([klog[b][max(n, 1) - 1] for b, n in enumerate(lens)])
+        vn = torch.stack([vlog[b][max(n, 1) - 1] for b, n in enumerate(lens)])
+        plan.flux_kv_append(layer, B, kn, vn, ktab, vtab, pos)
+        q = synth.normal_bf16((B, Hq, 128), 78, layer, DEV)
+        out = plan.flux_attn_decode(layer, B, q, ktab, vtab, ctx)
+        rec = plan.flux_debug_dispatch(B)
+        for b, n in enumerate(lens):
+            if n == 0:
+                assert torch.count_nonzero(out[b]) == 0
+                continue
+            mode = int(mask[b, layer])
+            ref = oracle.decode(mode, bits(q[b]), bits(klog[b]), bits(vlog[b]), n, S, W, _scale())
+            compare(out[b], ref, "decode b=%d n=%d mode=%d" % (b, n, mode))
+            rows = expand_ranges(rec[b])
+            want = oracle.kept(mode, n - 1, S, W).tolist()
+            if layout == 1 and mode == 0:
+                assert compact_rows_to_positions(rows, n, S, W) == want
+            else:
+                assert rows == want
+            assert rec[b, 0] == mode and rec[b, 2] == b
+    assert plan.flux_plan_status() == 0
+
+
+# ---- routing and error behaviour ---------------------------------------------------------------
+
+def test_router_inputs_and_device_flags(flux):
+    plan = _plan(flux, 3, 8, 2, 4, 8, 4, 64)
+    lg = np.array([[[1, 0], [0, 1], [2, 2]], [[-1, -1.5], [3, 3.5], [0, -0.0]]], dtype=np.float32)
+    want = oracle.route(lg)
+    assert np.array_equal(plan.flux_router_apply(logits=lg).cpu().numpy(), want)                       # host logits
+    assert np.array_equal(plan.flux_router_apply(logits=torch.from_numpy(lg).to(DEV)).cpu().numpy(), want)
+    assert plan.flux_plan_status() == 0
+    bad = lg.copy(); bad[1, 1, 0] = np.nan
+    with pytest.raises(flux.FluxError) as e:
+        plan.flux_router_apply(logits=bad)
+    assert e.value.code == flux.FLUX_E_INVALID_ARG
+    plan.flux_router_apply(logits=torch.from_numpy(bad).to(DEV))
+    assert plan.flux_plan_status(raise_on_flag=False) == flux.FLUX_STATUS_NAN_LOGIT
+    assert plan.flux_plan_status() == 0                        # reading clears the word
+    with pytest.raises(flux.FluxError):
+        plan.flux_router_apply(mask=np.array([[1, 0, 2]], dtype=np.uint8))
+    plan.flux_router_apply(mask=torch.tensor([[1, 0, 2]], dtype=torch.uint8, device=DEV))
+    assert plan.flux_plan_status(raise_on_flag=False) == flux.FLUX_STATUS_BAD_MASK
+
+
+def test_host_side_argument_errors_launch_nothing(flux):
+    plan = _plan(flux, 2, 8, 2, 4, 8, 2, 64)
+    q = torch.zeros((4, 8, 128), dtype=torch.bfloat16, device=DEV)
+    k = torch.zeros((4, 2, 128), dtype=torch.bfloat16, device=DEV)
+    n0 = plan.flux_launch_count()
+    with pytest.raises(flux.FluxError):                         # no routing decision yet
+        plan.flux_attn_prefill(0, 0, q, k, k, 0)
+    plan.flux_router_apply(mask=np.array([[1, 0], [0, 1]], dtype=np.uint8))
+    n1 = plan.flux_launch_count()
+    assert n1 == n0 + 1
+    for args in [(5, 0, q, k, k, 0), (0, 2, q, k, k, 0), (0, 0, q, k, k, 61), (0, 0, q, k, k, -1)]:
+        with pytest.raises(flux.FluxError):
+            plan.flux_attn_prefill(*args)
+    with pytest.raises(flux.FluxError):                         # misaligned pointer
+        plan.flux_attn_prefill(0, 0, q.view(-1)[1:1 + 8 * 128].view(1, 8, 128), k, k, 0)
+    with pytest.raises(flux.FluxError):                         # batch beyond the routed batch
+        plan.flux_attn_decode(0, 3, q, 0, 0, 0)
+    assert plan.flux_launch_count() == n1
+    out = plan.flux_attn_prefill(0, 0, q[:0], k, k, 0)          # Nq = 0: no-op success
+    assert out.shape[0] == 0 and plan.flux_launch_count() == n1
+    # a context length beyond max_context is flagged by the device and clamped
+    kc = torch.zeros((64, 2, 128), dtype=torch.bfloat16, device=DEV)
+    tab = flux.pointer_table([kc, kc], DEV)
+    ctx = torch.tensor([65, 3], dtype=torch.int32, device=DEV)
+    plan.flux_attn_decode(0, 2, torch.zeros((2, 8, 128), dtype=torch.bfloat16, device=DEV), tab, tab, ctx)
+    assert plan.flux_plan_status(raise_on_flag=False) == flux.FLUX_STATUS_BAD_LENGTH
+
+
+def test_decode_host_entry_point_matches_device_entry_point(flux):
+    Hq, Hkv, S, W, B, L = 8, 2, 4, 8, 3, 2
+    lens = [30, 9, 17]
+    plan = _plan(flux, L, Hq, Hkv, S, W, B, 64)
+    plan.flux_router_apply(mask=np.array([[1, 0], [0, 0], [1, 1]], dtype=np.uint8))
+    kc = [synth.normal_bf16((64, Hkv, 128), 5, b, DEV) for b in range(B)]
+    vc = [synth.normal_bf16((64, Hkv, 128), 6, b, DEV) for b in range(B)]
+    kc2 = [t.clone() for t in kc]; vc2 = [t.clone() for t in vc]
+    q = synth.normal_bf16((B, Hq, 128), 7, 0, "cpu").pin_memory()
+    kn = synth.normal_bf16((B, Hkv, 128), 7, 1, "cpu").pin_memory()
+    vn = synth.normal_bf16((B, Hkv, 128), 7, 2, "cpu").pin_memory()
+    pos = torch.tensor([n - 1 for n in lens], dtype=torch.int32, device=DEV)
+    ctx = torch.tensor(lens, dtype=torch.int32, device=DEV)
+    out_h = torch.empty((B, Hq, 128), dtype=torch.bfloat16).pin_memory()
+    for layer in range(L):
+        kt, vt = flux.pointer_table(kc, DEV), flux.pointer_table(vc, DEV)
+        plan.flux_attn_decode_host(layer, B, q, kn, vn, kt, vt, pos, ctx, out_h)
+        torch.cuda.synchronize()
+        kt2, vt2 = flux.pointer_table(kc2, DEV), flux.pointer_table(vc2, DEV)
+        plan.flux_kv_append(layer, B, kn.to(DEV), vn.to(DEV), kt2, vt2, pos)
+        out_d = plan.flux_attn_decode(layer, B, q.to(DEV), kt2, vt2, ctx)
+        assert torch.equal(out_d.cpu(), out_h)
