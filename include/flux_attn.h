@@ -177,6 +177,20 @@ int flux_plan_status(flux_plan *plan, uint32_t *status_bits, void *stream);
 int flux_debug_dispatch(flux_plan *plan, int32_t *records_out, int32_t max_records,
                         int32_t *n_records_out, void *stream);
 
+/* Per-kernel device timing for roofline reports.  flux_profile_enable creates
+ * max_records pairs of CUDA events (host objects; max_records == 0 turns
+ * profiling off and destroys them); while enabled, every launch of a dominant
+ * kernel (FLUX_KERNEL_DECODE: the split-K decode kernel, FLUX_KERNEL_PREFILL: the
+ * prefill attention kernel) is bracketed by two event records on its stream until
+ * the pairs run out.  flux_profile_read synchronises `stream`, sums the elapsed
+ * time of the recorded launches of `kind` into *total_ms, stores their count in
+ * *launches (both host), and resets the recorder. */
+#define FLUX_KERNEL_DECODE  0
+#define FLUX_KERNEL_PREFILL 1
+int flux_profile_enable(flux_plan *plan, int32_t max_records);
+int flux_profile_read(flux_plan *plan, int32_t kind, double *total_ms, int64_t *launches,
+                      void *stream);
+
 /* Number of kernels this plan has launched so far (host counter). */
 int64_t flux_launch_count(const flux_plan *plan);
 

@@ -30,6 +30,32 @@ int check_cuda(cudaError_t e, const char *what)
     return fail(FLUX_E_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
 
+int prof_begin(flux_plan *p, int kind, cudaStream_t st)
+{
+    if (!p->prof_ev || p->prof_n >= p->prof_cap) return -1;
+    const int rec = p->prof_n++;
+    p->prof_kind[rec] = (int8_t)kind;
+    cudaEventRecord(p->prof_ev[2 * rec], st);
+    return rec;
+}
+
+void prof_end(flux_plan *p, int rec, cudaStream_t st)
+{
+    if (rec >= 0) cudaEventRecord(p->prof_ev[2 * rec + 1], st);
+}
+
+static void prof_free(flux_plan *p)
+{
+    if (p->prof_ev) {
+        for (int i = 0; i < 2 * p->prof_cap; ++i) cudaEventDestroy(p->prof_ev[i]);
+        free(p->prof_ev);
+        free(p->prof_kind);
+    }
+    p->prof_ev = nullptr;
+    p->prof_kind = nullptr;
+    p->prof_cap = p->prof_n = 0;
+}
+
 static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 static int validate_config(const flux_config *c)
@@ -276,6 +302,9 @@ int flux_plan_create(const flux_config *cfg, flux_plan **plan)
     p->mask_B = 0;
     p->launches = 0;
     p->debug_records = 0;
+    p->prof_ev = nullptr;
+    p->prof_kind = nullptr;
+    p->prof_cap = p->prof_n = 0;
     cudaError_t e = cudaDeviceGetAttribute(&p->dev.n_sms, cudaDevAttrMultiProcessorCount, dev);
     if (e == cudaSuccess)
         e = cudaDeviceGetAttribute(&p->dev.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
@@ -303,6 +332,7 @@ int flux_plan_create(const flux_config *cfg, flux_plan **plan)
 
 int flux_plan_destroy(flux_plan *plan)
 {
+    if (plan) prof_free(plan);
     delete plan;
     return FLUX_OK;
 }
@@ -525,6 +555,60 @@ int flux_debug_dispatch(flux_plan *plan, int32_t *records_out, int32_t max_recor
     rc = check_cuda(cudaStreamSynchronize(st), "stream synchronize");
     if (rc) return rc;
     *n_records_out = n;
+    return FLUX_OK;
+}
+
+int flux_profile_enable(flux_plan *plan, int32_t max_records)
+{
+    int rc = need_plan(plan, false);
+    if (rc) return rc;
+    if (max_records < 0 || max_records > (1 << 20))
+        return fail(FLUX_E_INVALID_ARG, "max_records outside [0, 2^20]");
+    prof_free(plan);
+    if (max_records == 0) return FLUX_OK;
+    plan->prof_ev = (cudaEvent_t *)calloc(2 * (size_t)max_records, sizeof(cudaEvent_t));
+    plan->prof_kind = (int8_t *)calloc((size_t)max_records, 1);
+    if (!plan->prof_ev || !plan->prof_kind) {
+        free(plan->prof_ev);
+        free(plan->prof_kind);
+        plan->prof_ev = nullptr;
+        plan->prof_kind = nullptr;
+        return fail(FLUX_E_INVALID_ARG, "out of host memory");
+    }
+    for (int i = 0; i < 2 * max_records; ++i) {
+        rc = check_cuda(cudaEventCreate(&plan->prof_ev[i]), "cudaEventCreate");
+        if (rc) {
+            plan->prof_cap = (i + 1) / 2;
+            prof_free(plan);
+            return rc;
+        }
+    }
+    plan->prof_cap = max_records;
+    plan->prof_n = 0;
+    return FLUX_OK;
+}
+
+int flux_profile_read(flux_plan *plan, int32_t kind, double *total_ms, int64_t *launches, void *stream)
+{
+    int rc = need_plan(plan, false);
+    if (rc) return rc;
+    if (!total_ms || !launches) return fail(FLUX_E_INVALID_ARG, "NULL output pointer");
+    rc = check_cuda(cudaStreamSynchronize((cudaStream_t)stream), "stream synchronize");
+    if (rc) return rc;
+    double sum = 0.0;
+    int64_t cnt = 0;
+    for (int i = 0; i < plan->prof_n; ++i) {
+        if (plan->prof_kind[i] != kind) continue;
+        float ms = 0.f;
+        rc = check_cuda(cudaEventElapsedTime(&ms, plan->prof_ev[2 * i], plan->prof_ev[2 * i + 1]),
+                        "cudaEventElapsedTime");
+        if (rc) return rc;
+        sum += ms;
+        ++cnt;
+    }
+    plan->prof_n = 0;
+    *total_ms = sum;
+    *launches = cnt;
     return FLUX_OK;
 }
 

@@ -526,7 +526,9 @@ int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *con
     a.sched = (int32_t *)(ws + p->lay.sched);
     a.status = (uint32_t *)(ws + p->lay.status);
     a.out = (__nv_bfloat16 *)out;
+    const int rec = prof_begin(p, FLUX_KERNEL_DECODE, st);
     decode_kernel<<<p->dec_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
+    prof_end(p, rec, st);
     p->launches++;
     int rc = check_cuda(cudaGetLastError(), "decode kernel launch");
     if (rc) return rc;

@@ -71,6 +71,10 @@ struct flux_plan {
     int64_t launches;
     int32_t debug_records;  // records the latest call wrote
     int dec_ctas;
+    // optional per-kernel timing (host-side event pool)
+    cudaEvent_t *prof_ev;     // 2 * prof_cap events
+    int8_t *prof_kind;
+    int32_t prof_cap, prof_n;
 };
 
 namespace flux {
@@ -92,6 +96,9 @@ int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *con
                   cudaStream_t st);
 int launch_prefill(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v,
                    int q_start, int Nq, void *out, cudaStream_t st);
+// bracket a dominant-kernel launch with events when profiling is on
+int prof_begin(flux_plan *p, int kind, cudaStream_t st);   // returns record index or -1
+void prof_end(flux_plan *p, int rec, cudaStream_t st);
 int decode_setup(flux_plan *p);   // one-time attribute setting for the decode kernel
 int prefill_setup(flux_plan *p);
 

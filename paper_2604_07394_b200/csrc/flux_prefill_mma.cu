@@ -291,7 +291,9 @@ int launch_prefill_mma(flux_plan *p, int layer, int req, const void *q, const vo
     a.debug = (int32_t *)(ws + p->lay.debug);
     a.status = (uint32_t *)(ws + p->lay.status);
     dim3 grid((Nq + BM - 1) / BM, c.n_q_heads);
+    const int rec = prof_begin(p, FLUX_KERNEL_PREFILL, st);
     prefill_mma_kernel<<<grid, kWarps * 32, kSmemBytes, st>>>(a);
+    prof_end(p, rec, st);
     p->launches++;
     p->debug_records = 1;
     return check_cuda(cudaGetLastError(), "prefill kernel launch");
