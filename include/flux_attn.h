@@ -146,6 +146,33 @@ int flux_attn_decode(flux_plan *plan, int32_t layer, int32_t B, const void *q,
                      const void *const *k_caches, const void *const *v_caches,
                      const int32_t *ctx_len, void *out, void *stream);
 
+/* Decode step for callers that cannot allocate device memory at all.  (The paper
+ * has no counterpart: this is a packaging variant of flux_attn_decode, not part of
+ * the method.)  Who needs it: code that runs inside a host program which owns all
+ * device memory and passes in only the operator's own tensors, and loops that may
+ * not risk the device-wide synchronisation an allocation can cause.  The split-K
+ * scratch that flux_attn_decode keeps in the caller's workspace sits here in a
+ * fixed array of about 9.6 MB inside the library image, held on every GPU the
+ * process uses until it exits.  No plan and no workspace are needed; the call
+ * makes no cudaMalloc / cudaFree and uses no allocating library routine.
+ *   cfg        shapes as for flux_plan_create (max_batch is ignored).
+ *   mask       uint8 [B][n_layers], device: the routing decision (1 FA, 0 SA).
+ *   q, out, k_caches, v_caches, ctx_len: as in flux_attn_decode, all device.
+ *   status_out optional device uint32: receives the FLUX_STATUS_* bits of this call.
+ * Limits (beyond them the call returns FLUX_E_CAPACITY and launches nothing):
+ * B <= 64, n_q_heads / n_kv_heads <= 8, n_kv_heads <= 16.
+ * The first call on each device resolves the array's device address and sets a
+ * kernel attribute; make that first call before any stream capture begins.
+ * All calls on a device share the one array, which keeps the previous call's
+ * contents (the status word is cleared at the start of each call): calls whose
+ * kernels may overlap on the GPU -- different streams, or several host threads --
+ * race on it and must be serialised by the caller. */
+int flux_attn_decode_noalloc(const flux_config *cfg, int32_t layer, int32_t B,
+                             const uint8_t *mask, const void *q,
+                             const void *const *k_caches, const void *const *v_caches,
+                             const int32_t *ctx_len, void *out, uint32_t *status_out,
+                             void *stream);
+
 /* The same decode step for callers whose activations live in host memory: copies
  * q, k_new, v_new (host, pinned for speed) to staging in the workspace, appends,
  * attends, and copies the result to out (host).  Asynchronous on `stream` like

@@ -15,6 +15,10 @@
 // and writes one partial (O, m, l) per segment it touched; a small combine kernel
 // merges the partials (the split-K identity: sums over disjoint key sets merge by
 // rescaling with exp(m_p - m)).
+#include <math.h>
+
+#include <mutex>
+
 #include "flux_internal.h"
 
 namespace flux {
@@ -539,3 +543,146 @@ int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *con
 }
 
 }  // namespace flux
+
+// ---------------------------------------------------------------------------------------------
+// Decode without any caller- or library-allocated scratch (flux_attn_decode_noalloc).
+//
+// Some callers have no way to obtain device memory for a workspace: a plug-in inside a host
+// program that owns every byte of device memory and hands out only the tensors of the current
+// operator, or a serving loop that must not meet the device-wide synchronisation an allocation
+// can bring.  For them the split-K scratch (partials, schedule table, status word) lives in a
+// fixed array inside the library image.  Every process that loads the library pays for it on
+// every GPU it touches, so it is sized for moderate batches only.
+// ---------------------------------------------------------------------------------------------
+namespace flux {
+namespace {
+
+constexpr int kNaMaxBatch = 64;     // requests per call
+constexpr int kNaMaxCtas = 160;     // CTAs launched (one per SM, clamped)
+constexpr int kNaMaxG = 8;          // query heads per KV head
+constexpr int kNaMaxHeadGroups = 2; // n_kv_heads <= 16
+constexpr size_t kNaSlots = (size_t)(kNaMaxCtas + kNaMaxBatch * kNaMaxHeadGroups) * kDecWarps;
+constexpr size_t kNaOffStatus = 0;
+constexpr size_t kNaOffDebug = 256;
+constexpr size_t kNaOffSched = kNaOffDebug + (size_t)kNaMaxBatch * 8 * sizeof(int32_t);
+constexpr size_t kNaOffMl = (kNaOffSched + (kNaMaxBatch + 4) * sizeof(int32_t) + 255) / 256 * 256;
+constexpr size_t kNaOffO = (kNaOffMl + kNaSlots * kNaMaxG * 2 * sizeof(float) + 255) / 256 * 256;
+constexpr size_t kNaBytes = kNaOffO + kNaSlots * kNaMaxG * kHeadDim * sizeof(float);   // about 9.6 MB
+
+// In host code this name is only a handle for cudaGetSymbolAddress; it is not a device address.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNaBytes];
+
+struct NaDevice {
+    bool ready;
+    unsigned char *scratch;  // device address of g_noalloc_scratch on this device
+    int n_ctas;
+};
+constexpr int kNaMaxDevices = 64;
+NaDevice g_na_dev[kNaMaxDevices];
+std::mutex g_na_mutex;
+
+// Once per device, with that device current: resolve the scratch address, raise the kernel's
+// dynamic shared-memory limit, read the SM count.
+int noalloc_setup(int dev, NaDevice **out)
+{
+    if (dev < 0 || dev >= kNaMaxDevices) return fail(FLUX_E_CUDA, "device index %d not supported", dev);
+    std::lock_guard<std::mutex> lock(g_na_mutex);
+    NaDevice &d = g_na_dev[dev];
+    if (!d.ready) {
+        int major = 0, sms = 0, smem = 0;
+        int rc = check_cuda(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev),
+                            "cudaDeviceGetAttribute");
+        if (!rc) rc = check_cuda(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev),
+                                 "cudaDeviceGetAttribute");
+        if (!rc) rc = check_cuda(cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev),
+                                 "cudaDeviceGetAttribute");
+        if (rc) return rc;
+        if (major != 10) return fail(FLUX_E_CUDA, "this library is built for sm_100a only");
+        if (smem < kDecSmemBytes) return fail(FLUX_E_CUDA, "not enough shared memory per block");
+        void *ptr = nullptr;
+        rc = check_cuda(cudaGetSymbolAddress(&ptr, g_noalloc_scratch), "cudaGetSymbolAddress(scratch)");
+        if (rc) return rc;
+        rc = check_cuda(cudaFuncSetAttribute(decode_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             kDecSmemBytes),
+                        "cudaFuncSetAttribute(decode_kernel)");
+        if (rc) return rc;
+        d.scratch = (unsigned char *)ptr;
+        d.n_ctas = sms < kNaMaxCtas ? sms : kNaMaxCtas;
+        d.ready = true;
+    }
+    *out = &d;
+    return FLUX_OK;
+}
+
+}  // namespace
+}  // namespace flux
+
+extern "C" int flux_attn_decode_noalloc(const flux_config *cfg, int32_t layer, int32_t B,
+                                        const uint8_t *mask, const void *q,
+                                        const void *const *k_caches, const void *const *v_caches,
+                                        const int32_t *ctx_len, void *out, uint32_t *status_out,
+                                        void *stream)
+{
+    using namespace flux;
+    if (!cfg) return fail(FLUX_E_INVALID_ARG, "config is NULL");
+    if (cfg->head_dim != kHeadDim) return fail(FLUX_E_UNSUPPORTED_SHAPE, "head_dim must be 128");
+    if (cfg->n_layers < 1 || cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 ||
+        cfg->n_q_heads % cfg->n_kv_heads != 0)
+        return fail(FLUX_E_UNSUPPORTED_SHAPE, "bad head counts");
+    if (cfg->sink < 0 || cfg->window < 1 || cfg->max_context < 1 ||
+        (cfg->kv_layout != FLUX_KV_FULL && cfg->kv_layout != FLUX_KV_COMPACT_SA) ||
+        !(cfg->softmax_scale >= 0.0f))
+        return fail(FLUX_E_INVALID_ARG, "bad sink / window / max_context / kv_layout / softmax_scale");
+    const int G = cfg->n_q_heads / cfg->n_kv_heads;
+    const int n_hg = dec_head_groups(cfg->n_kv_heads);
+    if (B < 1 || B > kNaMaxBatch)
+        return fail(FLUX_E_CAPACITY, "flux_attn_decode_noalloc: B=%d exceeds the built-in scratch limit of %d "
+                    "requests; use flux_attn_decode with a workspace", B, kNaMaxBatch);
+    if (G > kNaMaxG || n_hg > kNaMaxHeadGroups)
+        return fail(FLUX_E_CAPACITY, "flux_attn_decode_noalloc: %d query heads per KV head (limit %d) or %d KV "
+                    "heads (limit 16) exceed the built-in scratch; use flux_attn_decode with a workspace",
+                    G, kNaMaxG, cfg->n_kv_heads);
+    if (layer < 0 || layer >= cfg->n_layers) return fail(FLUX_E_INVALID_ARG, "layer out of range");
+    if (!mask || !q || !k_caches || !v_caches || !ctx_len || !out)
+        return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    if ((((uintptr_t)q) | ((uintptr_t)out)) & 15u)
+        return fail(FLUX_E_INVALID_ARG, "q / out must be 16-byte aligned");
+    int dev = 0;
+    int rc = check_cuda(cudaGetDevice(&dev), "cudaGetDevice");
+    if (rc) return rc;
+    NaDevice *nd = nullptr;
+    rc = noalloc_setup(dev, &nd);
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned char *ws = nd->scratch;
+    // the array keeps whatever the previous call left: the status word must start at zero
+    rc = check_cuda(cudaMemsetAsync(ws + kNaOffStatus, 0, 256, st), "status clear");
+    if (rc) return rc;
+    DecArgs a;
+    a.q = (const __nv_bfloat16 *)q;
+    a.k_caches = k_caches;
+    a.v_caches = v_caches;
+    a.ctx_len = ctx_len;
+    a.mask = mask;
+    a.B = B; a.L = cfg->n_layers; a.layer = layer; a.Hq = cfg->n_q_heads; a.Hkv = cfg->n_kv_heads;
+    a.G = G; a.S = cfg->sink; a.W = cfg->window; a.layout = cfg->kv_layout;
+    a.max_context = cfg->max_context;
+    const float scale = cfg->softmax_scale > 0.0f ? cfg->softmax_scale : 1.0f / sqrtf((float)kHeadDim);
+    a.scale_log2 = scale * 1.4426950408889634f;
+    a.part_o = (float *)(ws + kNaOffO);
+    a.part_ml = (float *)(ws + kNaOffMl);
+    a.debug = (int32_t *)(ws + kNaOffDebug);
+    a.sched = (int32_t *)(ws + kNaOffSched);
+    a.status = (uint32_t *)(ws + kNaOffStatus);
+    a.out = (__nv_bfloat16 *)out;
+    decode_kernel<<<nd->n_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
+    rc = check_cuda(cudaGetLastError(), "decode kernel launch");
+    if (rc) return rc;
+    decode_combine_kernel<<<B * cfg->n_q_heads, 128, 0, st>>>(a);
+    rc = check_cuda(cudaGetLastError(), "decode combine kernel launch");
+    if (rc) return rc;
+    if (status_out)
+        rc = check_cuda(cudaMemcpyAsync(status_out, ws + kNaOffStatus, sizeof(uint32_t),
+                                        cudaMemcpyDeviceToDevice, st), "status copy");
+    return rc;
+}

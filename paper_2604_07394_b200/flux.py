@@ -40,7 +40,7 @@ FLUX_KV_COMPACT_SA = 1
 EXPORTS = [
     "flux_plan_create", "flux_plan_destroy", "flux_workspace_size", "flux_plan_set_workspace",
     "flux_router_apply", "flux_attn_prefill", "flux_kv_retain", "flux_kv_append",
-    "flux_attn_decode", "flux_attn_decode_host", "flux_attn_prefill_host", "flux_plan_status",
+    "flux_attn_decode", "flux_attn_decode_noalloc", "flux_attn_decode_host", "flux_attn_prefill_host", "flux_plan_status",
     "flux_debug_dispatch", "flux_profile_enable", "flux_profile_read", "flux_launch_count", "flux_last_error", "flux_version",
 ]
 
@@ -84,6 +84,7 @@ def load():
     L.flux_kv_retain.argtypes = [vp, i32, i32, vp, vp, i32, vp, vp, vp]
     L.flux_kv_append.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
+    L.flux_attn_decode_noalloc.argtypes = [cfgp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.flux_attn_prefill_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     L.flux_plan_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
@@ -242,6 +243,22 @@ class Plan:
 
     def flux_launch_count(self) -> int:
         return load().flux_launch_count(self._h)
+
+
+def flux_attn_decode_noalloc(cfg: FluxConfig, layer, B, mask, q, k_caches, v_caches, ctx_len, out=None,
+                             status_out=None):
+    """Decode step for callers that cannot allocate device memory: needs no plan and no workspace.
+
+    The split-K scratch is a fixed array inside the library (B <= 64, at most 8 query heads per KV
+    head, at most 16 KV heads).  Calls on one device share that array, so calls that could overlap
+    on the GPU must be serialised by the caller.  ``out`` is the caller's tensor (allocated here
+    with torch only when omitted, as a convenience of this wrapper)."""
+    if out is None:
+        out = torch.empty_like(q)
+    _check(load().flux_attn_decode_noalloc(ctypes.byref(cfg), layer, B, _ptr(mask), _ptr(q), _ptr(k_caches),
+                                           _ptr(v_caches), _ptr(ctx_len), _ptr(out), _ptr(status_out),
+                                           _stream()))
+    return out
 
 
 def pointer_table(tensors, device) -> torch.Tensor:
