@@ -218,6 +218,15 @@ int flux_profile_enable(flux_plan *plan, int32_t max_records);
 int flux_profile_read(flux_plan *plan, int32_t kind, double *total_ms, int64_t *launches,
                       void *stream);
 
+/* Which kernel flux_attn_prefill launches.  FLUX_PREFILL_AUTO (the default) and
+ * FLUX_PREFILL_TCGEN05 run the tcgen05 / TMEM / TMA kernel; FLUX_PREFILL_WARP_MMA runs
+ * the warp-level mma.sync kernel (kept for comparison).  Both compute Eq. 1 / Eq. 2 and
+ * serve every shape. */
+#define FLUX_PREFILL_AUTO     0
+#define FLUX_PREFILL_WARP_MMA 1
+#define FLUX_PREFILL_TCGEN05  2
+int flux_debug_prefill_kernel(flux_plan *plan, int32_t which);
+
 /* Number of kernels this plan has launched so far (host counter). */
 int64_t flux_launch_count(const flux_plan *plan);
 

@@ -419,6 +419,16 @@ int flux_attn_prefill(flux_plan *plan, int32_t layer, int32_t req, const void *q
     return launch_prefill(plan, layer, req, q, k, v, q_start, Nq, out, (cudaStream_t)stream);
 }
 
+int flux_debug_prefill_kernel(flux_plan *plan, int32_t which)
+{
+    int rc = need_plan(plan, false);
+    if (rc) return rc;
+    if (which < FLUX_PREFILL_AUTO || which > FLUX_PREFILL_TCGEN05)
+        return fail(FLUX_E_INVALID_ARG, "unknown prefill kernel selector %d", which);
+    plan->prefill_kernel = which;
+    return FLUX_OK;
+}
+
 int flux_kv_retain(flux_plan *plan, int32_t layer, int32_t req, const void *k_src, const void *v_src,
                    int32_t n, void *k_cache, void *v_cache, void *stream)
 {

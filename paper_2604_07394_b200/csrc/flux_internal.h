@@ -71,6 +71,7 @@ struct flux_plan {
     int64_t launches;
     int32_t debug_records;  // records the latest call wrote
     int dec_ctas;
+    int prefill_kernel;     // FLUX_PREFILL_*
     // optional per-kernel timing (host-side event pool)
     cudaEvent_t *prof_ev;     // 2 * prof_cap events
     int8_t *prof_kind;

@@ -1,4 +1,4 @@
-// Prefill dispatch: picks the kernel that serves a (shape, alignment) case.
+// Prefill dispatch: picks the kernel that serves a launch.
 #include "flux_internal.h"
 
 namespace flux {
@@ -6,17 +6,26 @@ namespace flux {
 int prefill_mma_setup();
 int launch_prefill_mma(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v,
                        int q_start, int Nq, void *out, cudaStream_t st);
+int prefill_tc_setup();
+int launch_prefill_tc(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v,
+                      int q_start, int Nq, void *out, cudaStream_t st);
 
 int prefill_setup(flux_plan *p)
 {
-    (void)p;
-    return prefill_mma_setup();
+    p->prefill_kernel = FLUX_PREFILL_AUTO;
+    int rc = prefill_mma_setup();
+    if (!rc) rc = prefill_tc_setup();
+    return rc;
 }
 
 int launch_prefill(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v,
                    int q_start, int Nq, void *out, cudaStream_t st)
 {
-    return launch_prefill_mma(p, layer, req, q, k, v, q_start, Nq, out, st);
+    // The tcgen05 kernel serves every shape (TMA zero-fills ragged tiles); the warp-MMA
+    // kernel stays selectable for comparison.
+    if (p->prefill_kernel == FLUX_PREFILL_WARP_MMA)
+        return launch_prefill_mma(p, layer, req, q, k, v, q_start, Nq, out, st);
+    return launch_prefill_tc(p, layer, req, q, k, v, q_start, Nq, out, st);
 }
 
 }  // namespace flux

@@ -1,0 +1,537 @@
+// Causal prefill of one routed layer on the sm_100a tensor cores (tcgen05 + TMEM + TMA).
+//
+// One CTA serves two query tiles at once: the same 128 query rows of two query
+// heads that share a KV head (GQA), so every K / V tile fetched by TMA feeds four
+// MMAs.  Roles (warp-specialised, 10 warps):
+//   warps 0-3   softmax of query tile 0 (one thread per query row, TMEM lane = row)
+//   warps 4-7   softmax of query tile 1
+//   warp  8     TMA producer: Q once, then K_j, V_j through a ring of shared-memory slots
+//   warp  9     MMA issuer: S = Q K^T (operands in shared memory), O += P V (P in TMEM)
+// TMEM (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; P (bf16) overwrites the
+// first 64 columns of its S.  The tensor pipe alternates between the two tiles, so the
+// softmax of one tile overlaps the MMAs of the other.  Softmax is the online form in
+// fp32 in the log2 domain; the running maximum is only raised when a tile exceeds it by
+// more than 2^8 (the accumulator and the row sum stay consistent with the maximum in
+// use, so the result is the same softmax), which makes rescaling O in TMEM rare.
+// An FA layer (Eq. 1) walks every KV tile up to the diagonal; an SA layer (Eq. 2 with the
+// streaming subset) walks the sink tiles and the window tiles only.
+//
+// Every mbarrier wait is bounded: when it runs out the CTA raises
+// FLUX_STATUS_WAIT_EXPIRED, stops issuing work, lets in-flight copies land, frees its
+// TMEM and returns; CTAs that start after that return at once.
+#include <cuda.h>
+
+#include "flux_internal.h"
+
+namespace flux {
+namespace {
+
+constexpr int BM = 128, BN = 128;
+constexpr int kHalfBytes = BM * 128;              // 128 rows x 64 bf16 (one 128-byte swizzle span per row)
+constexpr int kTileBytes = 2 * kHalfBytes;        // a 128 x 128 bf16 tile = two halves (d 0-63 | d 64-127)
+constexpr int kKvSlots = 4;
+constexpr int kThreads = 320;
+constexpr int kSoftmaxThreads = 128;
+
+constexpr int OFF_Q = 0;                          // Q tile 0, Q tile 1
+constexpr int OFF_KV = 2 * kTileBytes;
+constexpr int OFF_BAR = OFF_KV + kKvSlots * kTileBytes;
+constexpr int BAR_Q_FULL = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = 5, BAR_S_FULL = 9, BAR_P_FULL = 11,
+              BAR_O_FULL = 13, kNumBars = 15;
+constexpr int OFF_TMEM_PTR = OFF_BAR + 16 * 8;
+constexpr int OFF_ABORT = OFF_TMEM_PTR + 4;
+constexpr int kSmemBytes = OFF_BAR + 256 + 1024;  // + slack to align the base to 1024 bytes
+
+constexpr uint32_t kTmemCols = 512;
+constexpr uint32_t TM_S = 0, TM_O = 256;          // + 128 * tile
+
+constexpr long long kWaitCycles = 2000000000ll;   // bound of one mbarrier wait (about a second)
+constexpr float kRescaleThreshold = 8.0f;         // log2 units
+
+// instruction descriptor, kind::f16: D fp32, A and B bf16, M 128, N 128
+constexpr uint32_t kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+constexpr uint32_t kIdescQK = kIdescBase;               // A, B K-major
+constexpr uint32_t kIdescPV = kIdescBase | (1u << 16);  // B (= V) MN-major
+
+struct TcArgs {
+    __nv_bfloat16 *out;
+    const uint8_t *mask;
+    int L, layer, req, Hq, G, S, W, q_start, Nq;
+    int n_qt, ppg, n_pairs;
+    float scale_log2;
+    int32_t *debug;
+    uint32_t *status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+// ---- mbarrier ---------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the CTA is aborting or the limit ran out (which raises the flag).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          uint32_t *status)
+{
+    if (mbar_try(bar, parity)) return true;
+    const long long t0 = clock64();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycles) {
+            *abort_flag = 1;
+            atomicOr(status, FLUX_STATUS_WAIT_EXPIRED);
+            return false;
+        }
+    }
+}
+
+// ---- TMA ----------------------------------------------------------------------
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+                 ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+// ---- tcgen05 -------------------------------------------------------------------
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void tc_mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void tc_mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc, uint32_t acc)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+                 ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
+          "r"(taddr) : "memory");
+}
+
+// Shared-memory operand descriptor, 128-byte swizzle, 8-row groups 1024 bytes apart.
+// K-major operands (Q, K): leading offset unused.  MN-major operand (V): the leading
+// offset is the distance between the two 64-column halves of the tile.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes)
+{
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(1024u >> 4) << 32) |
+           (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ float fast_exp2(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// KV tile index of the it-th tile a query tile keeps: sink tiles [0, e1), then window tiles from b2
+__device__ __forceinline__ int tile_of(int it, int e1, int b2) { return it < e1 ? it : b2 + (it - e1); }
+
+__global__ void __launch_bounds__(kThreads, 1)
+prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                  const __grid_constant__ CUtensorMap tm_v, TcArgs a)
+{
+    extern __shared__ unsigned char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t sb = (raw + 1023u) & ~1023u;          // shared-window address of the aligned base
+    unsigned char *sm = smem_raw + (sb - raw);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sm + OFF_ABORT);
+    volatile uint32_t *tmem_ptr_smem = reinterpret_cast<volatile uint32_t *>(sm + OFF_TMEM_PTR);
+    const uint32_t bar0 = sb + OFF_BAR;
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // a CTA that starts after a wait has run out anywhere does nothing
+    if (tid == 0) *abort_flag = (*reinterpret_cast<volatile uint32_t *>(a.status) & FLUX_STATUS_WAIT_EXPIRED) ? 1 : 0;
+    __syncthreads();
+    if (*abort_flag) return;
+
+    // ---- which work item ----
+    const int bid = blockIdx.x;
+    const int qt = a.n_qt - 1 - bid / a.n_pairs;          // latest (heaviest) query tiles first
+    const int pr = bid % a.n_pairs;
+    const int kvh = pr / a.ppg, pi = pr % a.ppg;
+    const int h0 = kvh * a.G + 2 * pi;
+    const int nslots = (2 * pi + 1 < a.G) ? 2 : 1;
+    const int q_end = a.q_start + a.Nq;                   // KV rows present
+    const int i0 = a.q_start + qt * BM;
+    const int i_hi = min(i0 + BM - 1, q_end - 1);
+
+    const uint8_t mode_raw = a.mask[a.req * a.L + a.layer];
+    if (mode_raw > 1 && tid == 0) atomicOr(a.status, FLUX_STATUS_BAD_MASK);
+    const bool fa = mode_raw != 0;
+    const int S = a.S, W = a.W;
+
+    if (bid == 0 && tid == 0) {
+        const int n = q_end;
+        const bool two = !fa && n > S + W;
+        int32_t *d = a.debug;
+        d[0] = fa ? 1 : 0; d[1] = a.layer; d[2] = a.req; d[3] = n;
+        d[4] = 0; d[5] = two ? S : n; d[6] = two ? n - W : 0; d[7] = two ? n : 0;
+    }
+
+    int e1, b2;
+    const int e2 = i_hi / BN + 1;
+    if (fa) {
+        e1 = 0;
+        b2 = 0;
+    } else {
+        e1 = min((S + BN - 1) / BN, e2);
+        b2 = max(e1, max(0, i0 - W + 1) / BN);
+    }
+    const int n_tiles = e1 + max(0, e2 - b2);
+
+    // ---- set-up: barriers, TMEM ----
+    if (tid == 0) {
+        mbar_init(bar(BAR_Q_FULL), 1);
+        for (int s = 0; s < kKvSlots; ++s) {
+            mbar_init(bar(BAR_KV_FULL + s), 1);
+            mbar_init(bar(BAR_KV_EMPTY + s), 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(bar(BAR_S_FULL + t), 1);
+            mbar_init(bar(BAR_P_FULL + t), kSoftmaxThreads);
+            mbar_init(bar(BAR_O_FULL + t), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 9) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(sb + OFF_TMEM_PTR), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_ptr_smem;
+
+    if (warp == 8) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            mbar_expect_tx(bar(BAR_Q_FULL), (uint32_t)(nslots * kTileBytes));
+            for (int t = 0; t < nslots; ++t) {
+                tma_load_3d(sb + OFF_Q + t * kTileBytes, &tm_q, bar(BAR_Q_FULL), 0, h0 + t, qt * BM);
+                tma_load_3d(sb + OFF_Q + t * kTileBytes + kHalfBytes, &tm_q, bar(BAR_Q_FULL), 64, h0 + t, qt * BM);
+            }
+            bool ok = true;
+            for (int it = 0; it < n_tiles && ok; ++it) {
+                const int j0 = tile_of(it, e1, b2) * BN;
+#pragma unroll
+                for (int kv = 0; kv < 2; ++kv) {
+                    const int qi = 2 * it + kv, slot = qi & (kKvSlots - 1), use = qi / kKvSlots;
+                    ok = mbar_wait(bar(BAR_KV_EMPTY + slot), (uint32_t)((use & 1) ^ 1), abort_flag, a.status);
+                    if (!ok) break;
+                    const uint32_t dst = sb + OFF_KV + slot * kTileBytes;
+                    const CUtensorMap *tm = kv ? &tm_v : &tm_k;
+                    mbar_expect_tx(bar(BAR_KV_FULL + slot), (uint32_t)kTileBytes);
+                    tma_load_3d(dst, tm, bar(BAR_KV_FULL + slot), 0, kvh, j0);
+                    tma_load_3d(dst + kHalfBytes, tm, bar(BAR_KV_FULL + slot), 64, kvh, j0);
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 9) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            auto qk = [&](int t, int slot) {   // S_t = Q_t K^T
+                const uint32_t qb = sb + OFF_Q + t * kTileBytes, kb = sb + OFF_KV + slot * kTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const uint32_t off = (uint32_t)((kk >> 2) * kHalfBytes + (kk & 3) * 32);
+                    tc_mma_ss(tmem + TM_S + t * 128, smem_desc(qb + off, 16), smem_desc(kb + off, 16), kIdescQK,
+                              kk > 0 ? 1u : 0u);
+                }
+            };
+            auto pv = [&](int t, int slot, bool acc) {   // O_t (+)= P_t V
+                const uint32_t vb = sb + OFF_KV + slot * kTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    tc_mma_ts(tmem + TM_O + t * 128, tmem + TM_S + t * 128 + kk * 8,
+                              smem_desc(vb + kk * 2048, kHalfBytes), kIdescPV, (acc || kk > 0) ? 1u : 0u);
+            };
+            bool ok = mbar_wait(bar(BAR_Q_FULL), 0, abort_flag, a.status);
+            if (ok) ok = mbar_wait(bar(BAR_KV_FULL + 0), 0, abort_flag, a.status);
+            if (ok) {
+                tc_fence_after();
+                for (int t = 0; t < nslots; ++t) {
+                    qk(t, 0);
+                    tc_commit(bar(BAR_S_FULL + t));
+                }
+                tc_commit(bar(BAR_KV_EMPTY + 0));
+            }
+            for (int it = 0; it < n_tiles && ok; ++it) {
+                const int vq = 2 * it + 1, vslot = vq & (kKvSlots - 1), vpar = (vq / kKvSlots) & 1;
+                const int kq = 2 * it + 2, kslot = kq & (kKvSlots - 1), kpar = (kq / kKvSlots) & 1;
+                const bool more = it + 1 < n_tiles;
+                ok = mbar_wait(bar(BAR_KV_FULL + vslot), (uint32_t)vpar, abort_flag, a.status);
+                for (int t = 0; t < nslots && ok; ++t) {
+                    ok = mbar_wait(bar(BAR_P_FULL + t), (uint32_t)(it & 1), abort_flag, a.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    pv(t, vslot, it > 0);
+                    if (t == nslots - 1) tc_commit(bar(BAR_KV_EMPTY + vslot));
+                    if (more) {
+                        if (t == 0) {
+                            ok = mbar_wait(bar(BAR_KV_FULL + kslot), (uint32_t)kpar, abort_flag, a.status);
+                            if (!ok) break;
+                            tc_fence_after();
+                        }
+                        qk(t, kslot);
+                        tc_commit(bar(BAR_S_FULL + t));
+                        if (t == nslots - 1) tc_commit(bar(BAR_KV_EMPTY + kslot));
+                    } else {
+                        tc_commit(bar(BAR_O_FULL + t));
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp < 4 * nslots) {
+        // ================= softmax of query tile t =================
+        const int t = warp >> 2;
+        const int r = tid & 127;                         // row of the tile = TMEM lane
+        const int row = i0 + r;                          // absolute position of this query
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_base + TM_S + t * 128;
+        const uint32_t tO = tmem + lane_base + TM_O + t * 128;
+        float m_used = -INFINITY;                        // running maximum in use, scaled log2 units
+        float l = 0.f;
+        bool ok = true;
+        for (int it = 0; it < n_tiles; ++it) {
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_FULL + t), (uint32_t)(it & 1), abort_flag, a.status));
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t sr[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tc_ld32(tS + c * 32, sr[c]);
+            tc_wait_ld();
+            const int j0 = tile_of(it, e1, b2) * BN;
+            const int jmax = j0 + BN - 1;
+            const bool full = (jmax <= i0) && (fa || jmax < S || j0 > i0 + BM - 1 - W);
+            if (!full) {
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const int key = j0 + c * 32 + e;
+                        const bool keep = key <= row && (fa || key < S || key > row - W);
+                        if (!keep) sr[c][e] = 0xff800000u;   // -inf
+                    }
+            }
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+            for (int e = 0; e < 32; ++e) {
+                mx0 = fmaxf(mx0, __uint_as_float(sr[0][e]));
+                mx1 = fmaxf(mx1, __uint_as_float(sr[1][e]));
+                mx2 = fmaxf(mx2, __uint_as_float(sr[2][e]));
+                mx3 = fmaxf(mx3, __uint_as_float(sr[3][e]));
+            }
+            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;
+            const bool need = mx > m_used + kRescaleThreshold;
+            if (__any_sync(0xffffffffu, need)) {
+                const float alpha = need ? fast_exp2(m_used - mx) : 1.0f;   // 0 when nothing was kept so far
+                if (need) m_used = mx;
+                l *= alpha;
+                if (it > 0) {
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t o[32];
+                        tc_ld32(tO + c * 32, o);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        tc_st32(tO + c * 32, o);
+                    }
+                }
+            }
+            const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t p[32];
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    const float a0 = fast_exp2(fmaf(__uint_as_float(sr[2 * c][2 * e]), a.scale_log2, neg_m));
+                    const float a1 = fast_exp2(fmaf(__uint_as_float(sr[2 * c][2 * e + 1]), a.scale_log2, neg_m));
+                    const float b0 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1][2 * e]), a.scale_log2, neg_m));
+                    const float b1 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1][2 * e + 1]), a.scale_log2, neg_m));
+                    l0 += a0; l1 += a1; l2 += b0; l3 += b1;
+                    p[e] = pack_bf16(a0, a1);
+                    p[16 + e] = pack_bf16(b0, b1);
+                }
+                tc_st32(tS + c * 32, p);                 // P columns [32c, 32c+32) = keys [64c, 64c+64)
+            }
+            l += (l0 + l1) + (l2 + l3);
+            tc_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar(BAR_P_FULL + t));
+        }
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_O_FULL + t), 0, abort_flag, a.status));
+        if (ok) {
+            tc_fence_after();
+            const float inv = 1.0f / l;
+            const bool valid = row < q_end;
+            __nv_bfloat16 *dst = a.out + ((size_t)(valid ? row - a.q_start : 0) * a.Hq + (h0 + t)) * kHeadDim;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t o[32];
+                tc_ld32(tO + c * 32, o);
+                tc_wait_ld();
+                if (valid) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        uint4 w;
+                        w.x = pack_bf16(__uint_as_float(o[8 * e + 0]) * inv, __uint_as_float(o[8 * e + 1]) * inv);
+                        w.y = pack_bf16(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv);
+                        w.z = pack_bf16(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv);
+                        w.w = pack_bf16(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv);
+                        *reinterpret_cast<uint4 *>(dst + c * 32 + e * 8) = w;
+                    }
+                }
+            }
+        }
+    }
+
+    // ---- teardown ----
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // let copies and MMAs that were already issued land before the shared memory and TMEM go away
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+    if (warp == 9) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+// [rows][heads][128] bf16 tensor viewed as (d, head, row); box = 64 columns x 1 head x 128 rows
+int make_map(CUtensorMap *tm, const void *base, int heads, int rows)
+{
+    cuuint64_t dims[3] = {(cuuint64_t)kHeadDim, (cuuint64_t)heads, (cuuint64_t)rows};
+    cuuint64_t strides[2] = {(cuuint64_t)kRowBytes, (cuuint64_t)kRowBytes * (cuuint64_t)heads};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)BM};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(FLUX_E_CUDA, "cuTensorMapEncodeTiled failed with code %d", (int)r);
+    return FLUX_OK;
+}
+
+}  // namespace
+
+int prefill_tc_setup()
+{
+    if (!g_encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        int rc = check_cuda(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres),
+                            "cudaGetDriverEntryPointByVersion(cuTensorMapEncodeTiled)");
+        if (rc) return rc;
+        if (qres != cudaDriverEntryPointSuccess || !fn)
+            return fail(FLUX_E_CUDA, "the driver does not export cuTensorMapEncodeTiled");
+        g_encode = (EncodeTiledFn)fn;
+    }
+    return check_cuda(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes),
+                      "cudaFuncSetAttribute(prefill_tc_kernel)");
+}
+
+int launch_prefill_tc(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v, int q_start,
+                      int Nq, void *out, cudaStream_t st)
+{
+    const flux_config &c = p->cfg;
+    char *ws = (char *)p->ws;
+    CUtensorMap tq, tk, tv;
+    int rc = make_map(&tq, q, c.n_q_heads, Nq);
+    if (!rc) rc = make_map(&tk, k, c.n_kv_heads, q_start + Nq);
+    if (!rc) rc = make_map(&tv, v, c.n_kv_heads, q_start + Nq);
+    if (rc) return rc;
+    TcArgs a;
+    a.out = (__nv_bfloat16 *)out;
+    a.mask = p->d_mask;
+    a.L = c.n_layers; a.layer = layer; a.req = req; a.Hq = c.n_q_heads; a.G = p->G;
+    a.S = c.sink; a.W = c.window; a.q_start = q_start; a.Nq = Nq;
+    a.n_qt = (Nq + BM - 1) / BM;
+    a.ppg = (p->G + 1) / 2;
+    a.n_pairs = a.ppg * c.n_kv_heads;
+    a.scale_log2 = p->scale_log2;
+    a.debug = (int32_t *)(ws + p->lay.debug);
+    a.status = (uint32_t *)(ws + p->lay.status);
+    const int rec = prof_begin(p, FLUX_KERNEL_PREFILL, st);
+    prefill_tc_kernel<<<a.n_qt * a.n_pairs, kThreads, kSmemBytes, st>>>(tq, tk, tv, a);
+    prof_end(p, rec, st);
+    p->launches++;
+    p->debug_records = 1;
+    return check_cuda(cudaGetLastError(), "prefill tensor-core kernel launch");
+}
+
+}  // namespace flux

@@ -123,13 +123,17 @@ PREFILL_CASES = [
     (257, 8, 2, 0, 64, None),
     (400, 8, 8, 70, 129, (0, 100, 164, 400)),
     (520, 4, 1, 64, 256, (0, 512, 520)),
+    (777, 6, 2, 130, 300, (0, 1, 129, 500, 777)),
+    (1000, 3, 1, 0, 200, (0, 384, 1000)),
 ]
 
 
+@pytest.mark.parametrize("kernel", [2, 1], ids=["tcgen05", "warp_mma"])
 @pytest.mark.parametrize("N,Hq,Hkv,S,W,chunks", PREFILL_CASES)
-def test_prefill_small_shapes(flux, N, Hq, Hkv, S, W, chunks):
+def test_prefill_small_shapes(flux, N, Hq, Hkv, S, W, chunks, kernel):
     plan = _plan(flux, 2, Hq, Hkv, S, W, 1, 1024)
     plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
+    plan.flux_debug_prefill_kernel(kernel)
     seed = 1000 + N
     q = synth.normal_bf16((N, Hq, 128), seed, 1, DEV)
     k = synth.normal_bf16((N, Hkv, 128), seed, 2, DEV)
