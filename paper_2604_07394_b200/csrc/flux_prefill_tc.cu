@@ -2,11 +2,15 @@
 //
 // One CTA serves two query tiles at once: the same 128 query rows of two query
 // heads that share a KV head (GQA), so every K / V tile fetched by TMA feeds four
-// MMAs.  Roles (warp-specialised, 10 warps):
+// MMAs.  Roles (warp-specialised, three warpgroups):
 //   warps 0-3   softmax of query tile 0 (one thread per query row, TMEM lane = row)
 //   warps 4-7   softmax of query tile 1
 //   warp  8     TMA producer: Q once, then K_j, V_j through a ring of shared-memory slots
 //   warp  9     MMA issuer: S = Q K^T (operands in shared memory), O += P V (P in TMEM)
+//   warps 10-11 idle (they complete the third warpgroup, whose registers go to the softmax)
+// Registers are rebalanced per warpgroup (setmaxnreg works on whole warpgroups and inside
+// the CTA's own allocation): the third warpgroup shrinks to kOtherRegs, the two softmax
+// warpgroups grow to kSoftmaxRegs; the host checks that the CTA's allocation covers that.
 // TMEM (512 columns): S0 | S1 | O0 | O1, 128 fp32 columns each; P (bf16) overwrites the
 // first 64 columns of its S.  The tensor pipe alternates between the two tiles, so the
 // softmax of one tile overlaps the MMAs of the other.  Softmax is the online form in
@@ -30,8 +34,9 @@ constexpr int BM = 128, BN = 128;
 constexpr int kHalfBytes = BM * 128;              // 128 rows x 64 bf16 (one 128-byte swizzle span per row)
 constexpr int kTileBytes = 2 * kHalfBytes;        // a 128 x 128 bf16 tile = two halves (d 0-63 | d 64-127)
 constexpr int kKvSlots = 4;
-constexpr int kThreads = 320;
+constexpr int kThreads = 384;
 constexpr int kSoftmaxThreads = 128;
+constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // per-thread register targets after rebalancing
 
 constexpr int OFF_Q = 0;                          // Q tile 0, Q tile 1
 constexpr int OFF_KV = 2 * kTileBytes;
@@ -268,6 +273,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     tc_fence_after();
     const uint32_t tmem = *tmem_ptr_smem;
 
+    if (warp >= 8) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
     if (warp == 8) {
         // ================= TMA producer =================
         if (lane == 0) {
@@ -349,7 +356,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             }
         }
         __syncwarp();
-    } else if (warp < 4 * nslots) {
+    }
+    } else {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
+    if (warp < 4 * nslots) {   // (the softmax warps of an unused tile fall through)
         // ================= softmax of query tile t =================
         const int t = warp >> 2;
         const int r = tid & 127;                         // row of the tile = TMEM lane
@@ -455,6 +465,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         }
     }
 
+    }
+
     // ---- teardown ----
     tc_fence_before();
     __syncthreads();
@@ -501,6 +513,14 @@ int prefill_tc_setup()
             return fail(FLUX_E_CUDA, "the driver does not export cuTensorMapEncodeTiled");
         g_encode = (EncodeTiledFn)fn;
     }
+    // setmaxnreg moves registers inside the CTA's own allocation (registers per thread at launch x
+    // threads); a request beyond it would block for ever, so refuse to run rather than launch that.
+    cudaFuncAttributes fa;
+    int rc = check_cuda(cudaFuncGetAttributes(&fa, prefill_tc_kernel), "cudaFuncGetAttributes(prefill_tc_kernel)");
+    if (rc) return rc;
+    if (fa.numRegs * kThreads < 2 * kSoftmaxThreads * kSoftmaxRegs + (kThreads - 2 * kSoftmaxThreads) * kOtherRegs)
+        return fail(FLUX_E_CUDA, "prefill kernel was built with %d registers per thread: too few for its register rebalancing",
+                    fa.numRegs);
     return check_cuda(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes),
                       "cudaFuncSetAttribute(prefill_tc_kernel)");
 }
