@@ -17,6 +17,8 @@
 // fp32 in the log2 domain; the running maximum is only raised when a tile exceeds it by
 // more than 2^8 (the accumulator and the row sum stay consistent with the maximum in
 // use, so the result is the same softmax), which makes rescaling O in TMEM rare.
+// P is handed to the MMA issuer in two halves of 64 keys, so the first half of PV overlaps
+// the exponentials of the second.
 // An FA layer (Eq. 1) walks every KV tile up to the diagonal; an SA layer (Eq. 2 with the
 // streaming subset) walks the sink tiles and the window tiles only.
 //
@@ -41,9 +43,10 @@ constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // per-thread register targ
 constexpr int OFF_Q = 0;                          // Q tile 0, Q tile 1
 constexpr int OFF_KV = 2 * kTileBytes;
 constexpr int OFF_BAR = OFF_KV + kKvSlots * kTileBytes;
+// mbarriers: Q_FULL | KV_FULL[4] | KV_EMPTY[4] | S_FULL[2] | P_FULL[tile][half] | O_FULL[2]
 constexpr int BAR_Q_FULL = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = 5, BAR_S_FULL = 9, BAR_P_FULL = 11,
-              BAR_O_FULL = 13, kNumBars = 15;
-constexpr int OFF_TMEM_PTR = OFF_BAR + 16 * 8;
+              BAR_O_FULL = 15;
+constexpr int OFF_TMEM_PTR = OFF_BAR + 24 * 8;
 constexpr int OFF_ABORT = OFF_TMEM_PTR + 4;
 constexpr int kSmemBytes = OFF_BAR + 256 + 1024;  // + slack to align the base to 1024 bytes
 
@@ -109,6 +112,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             return false;
         }
     }
+}
+
+// One lane of a converged warp; the same lane every time for the same mask.  The producer and
+// issuer roles keep their control flow and address arithmetic warp-uniform and predicate only the
+// issuing instructions on this lane, so descriptors and addresses can stay in uniform registers.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred P;\n\telect.sync _|P, 0xffffffff;\n\tselp.u32 %0, 1, 0, P;\n\t}" : "=r"(pred));
+    return pred != 0;
 }
 
 // ---- TMA ----------------------------------------------------------------------
@@ -183,6 +196,30 @@ __device__ __forceinline__ float fast_exp2(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float fmax3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// packed pairs of fp32 (one instruction for two lanes of the FMA pipe)
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c)
+{
+    float2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;"
+        : "=l"(reinterpret_cast<uint64_t &>(d))
+        : "l"(reinterpret_cast<uint64_t const &>(a)), "l"(reinterpret_cast<uint64_t const &>(b)),
+          "l"(reinterpret_cast<uint64_t const &>(c)));
+    return d;
+}
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b)
+{
+    float2 d;
+    asm("add.f32x2 %0, %1, %2;"
+        : "=l"(reinterpret_cast<uint64_t &>(d))
+        : "l"(reinterpret_cast<uint64_t const &>(a)), "l"(reinterpret_cast<uint64_t const &>(b)));
+    return d;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     uint32_t r;
@@ -193,290 +230,325 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 // KV tile index of the it-th tile a query tile keeps: sink tiles [0, e1), then window tiles from b2
 __device__ __forceinline__ int tile_of(int it, int e1, int b2) { return it < e1 ? it : b2 + (it - e1); }
 
+// Per-CTA constants shared by the three roles.
+struct Cta {
+    uint32_t sb;            // shared-window address of the 1024-byte aligned base
+    uint32_t bar0;          // first mbarrier
+    uint32_t tmem;          // TMEM base address
+    volatile int *abort_flag;
+    uint32_t *status;
+    int qt, kvh, h0, nslots, q_end, i0;
+    int e1, b2, n_tiles;    // KV tiles kept: [0, e1) and [b2, b2 + n_tiles - e1)
+    bool fa;
+    __device__ __forceinline__ uint32_t bar(int i) const { return bar0 + 8u * (uint32_t)i; }
+    // every lane of the (converged) calling warp waits; the result is the same for all of them
+    __device__ __forceinline__ bool wait(int i, uint32_t parity) const
+    {
+        return __all_sync(0xffffffffu, mbar_wait(bar(i), parity, abort_flag, status));
+    }
+};
+
+// ================= TMA producer (one warp, one issuing lane) =================
+__device__ __forceinline__ void role_load(const Cta &c, const CUtensorMap *tm_q, const CUtensorMap *tm_k,
+                                          const CUtensorMap *tm_v)
+{
+    if (elect_one()) {
+        mbar_expect_tx(c.bar(BAR_Q_FULL), (uint32_t)(c.nslots * kTileBytes));
+        for (int t = 0; t < c.nslots; ++t) {
+            tma_load_3d(c.sb + OFF_Q + t * kTileBytes, tm_q, c.bar(BAR_Q_FULL), 0, c.h0 + t, c.qt * BM);
+            tma_load_3d(c.sb + OFF_Q + t * kTileBytes + kHalfBytes, tm_q, c.bar(BAR_Q_FULL), 64, c.h0 + t, c.qt * BM);
+        }
+    }
+    for (int it = 0; it < c.n_tiles; ++it) {
+        const int j0 = tile_of(it, c.e1, c.b2) * BN;
+#pragma unroll
+        for (int kv = 0; kv < 2; ++kv) {
+            const int qi = 2 * it + kv, slot = qi & (kKvSlots - 1), use = qi / kKvSlots;
+            if (!c.wait(BAR_KV_EMPTY + slot, (uint32_t)((use & 1) ^ 1))) return;
+            const uint32_t dst = c.sb + OFF_KV + slot * kTileBytes;
+            const CUtensorMap *tm = kv ? tm_v : tm_k;
+            if (elect_one()) {
+                mbar_expect_tx(c.bar(BAR_KV_FULL + slot), (uint32_t)kTileBytes);
+                tma_load_3d(dst, tm, c.bar(BAR_KV_FULL + slot), 0, c.kvh, j0);
+                tma_load_3d(dst + kHalfBytes, tm, c.bar(BAR_KV_FULL + slot), 64, c.kvh, j0);
+            }
+        }
+    }
+}
+
+// ================= MMA issuer (one warp, one issuing lane) =================
+// Issue order per KV tile j:  PV_0[j] QK_0[j+1] PV_1[j] QK_1[j+1]; the tensor pipe runs them in
+// that order, so S_t[j+1] overwrites S_t / P_t only after PV_t[j] has read P_t[j].
+__device__ __forceinline__ void role_mma(const Cta &c)
+{
+    // S_t = Q_t K^T, then up to two commits (tcgen05.commit belongs to the issuing lane; 0 = none)
+    auto qk = [&](int t, int slot, uint32_t bar_a, uint32_t bar_b) {
+        const uint32_t qb = c.sb + OFF_Q + t * kTileBytes, kb = c.sb + OFF_KV + slot * kTileBytes;
+        if (elect_one()) {
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const uint32_t off = (uint32_t)((kk >> 2) * kHalfBytes + (kk & 3) * 32);
+                tc_mma_ss(c.tmem + TM_S + t * 128, smem_desc(qb + off, 16), smem_desc(kb + off, 16), kIdescQK,
+                          kk > 0 ? 1u : 0u);
+            }
+            tc_commit(bar_a);
+            if (bar_b) tc_commit(bar_b);
+        }
+    };
+    // O_t (+)= P_t[:, 64 half ..] V[64 half ..]
+    auto pv_half = [&](int t, int slot, int half, bool acc, uint32_t bar_a, uint32_t bar_b) {
+        const uint32_t vb = c.sb + OFF_KV + slot * kTileBytes;
+        if (elect_one()) {
+#pragma unroll
+            for (int k4 = 0; k4 < 4; ++k4) {
+                const int kk = half * 4 + k4;
+                tc_mma_ts(c.tmem + TM_O + t * 128, c.tmem + TM_S + t * 128 + kk * 8,
+                          smem_desc(vb + kk * 2048, kHalfBytes), kIdescPV, (acc || kk > 0) ? 1u : 0u);
+            }
+            if (bar_a) tc_commit(bar_a);
+            if (bar_b) tc_commit(bar_b);
+        }
+    };
+    if (!c.wait(BAR_Q_FULL, 0)) return;
+    if (!c.wait(BAR_KV_FULL + 0, 0)) return;
+    tc_fence_after();
+    for (int t = 0; t < c.nslots; ++t)
+        qk(t, 0, c.bar(BAR_S_FULL + t), t == c.nslots - 1 ? c.bar(BAR_KV_EMPTY + 0) : 0u);
+    for (int it = 0; it < c.n_tiles; ++it) {
+        const int vq = 2 * it + 1, vslot = vq & (kKvSlots - 1), vpar = (vq / kKvSlots) & 1;
+        const int kq = 2 * it + 2, kslot = kq & (kKvSlots - 1), kpar = (kq / kKvSlots) & 1;
+        const bool more = it + 1 < c.n_tiles;
+        if (!c.wait(BAR_KV_FULL + vslot, (uint32_t)vpar)) return;
+        for (int t = 0; t < c.nslots; ++t) {
+            const bool last = t == c.nslots - 1;
+            if (!c.wait(BAR_P_FULL + 2 * t, (uint32_t)(it & 1))) return;
+            tc_fence_after();
+            pv_half(t, vslot, 0, it > 0, 0u, 0u);
+            if (!c.wait(BAR_P_FULL + 2 * t + 1, (uint32_t)(it & 1))) return;
+            tc_fence_after();
+            // after the second half: V slot free once the last tile's PV is done; O complete on the last KV tile
+            pv_half(t, vslot, 1, it > 0, more ? (last ? c.bar(BAR_KV_EMPTY + vslot) : 0u) : c.bar(BAR_O_FULL + t), 0u);
+            if (more) {
+                if (t == 0) {
+                    if (!c.wait(BAR_KV_FULL + kslot, (uint32_t)kpar)) return;
+                    tc_fence_after();
+                }
+                qk(t, kslot, c.bar(BAR_S_FULL + t), last ? c.bar(BAR_KV_EMPTY + kslot) : 0u);
+            }
+        }
+    }
+}
+
+// ================= softmax of query tile t (one thread per query row) =================
+__device__ __forceinline__ void role_softmax(const Cta &c, const TcArgs &a, int t, int warp, int lane)
+{
+    const int r = (warp & 3) * 32 + lane;            // row of the tile = TMEM lane
+    const int row = c.i0 + r;                        // absolute position of this query
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const uint32_t tS = c.tmem + lane_base + TM_S + t * 128;
+    const uint32_t tO = c.tmem + lane_base + TM_O + t * 128;
+    const int S = a.S, W = a.W;
+    const float scale_log2 = a.scale_log2;
+    float m_used = -INFINITY;                        // running maximum in use, scaled log2 units
+    float2 lsum = make_float2(0.f, 0.f);
+    for (int it = 0; it < c.n_tiles; ++it) {
+        if (!c.wait(BAR_S_FULL + t, (uint32_t)(it & 1))) return;
+        tc_fence_after();
+        uint32_t sr[4][32];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) tc_ld32(tS + q * 32, sr[q]);
+        tc_wait_ld();
+        const int j0 = tile_of(it, c.e1, c.b2) * BN;
+        const int jmax = j0 + BN - 1;
+        const bool full = (jmax <= c.i0) && (c.fa || jmax < S || j0 > c.i0 + BM - 1 - W);
+        if (!full) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int e = 0; e < 32; ++e) {
+                    const int key = j0 + q * 32 + e;
+                    const bool keep = key <= row && (c.fa || key < S || key > row - W);
+                    if (!keep) sr[q][e] = 0xff800000u;   // -inf
+                }
+        }
+        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+#pragma unroll
+            for (int e = 0; e < 32; e += 2)
+                mx[q] = fmax3(mx[q], __uint_as_float(sr[q][e]), __uint_as_float(sr[q][e + 1]));
+        const float mxs = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;
+        const bool need = mxs > m_used + kRescaleThreshold;
+        if (__any_sync(0xffffffffu, need)) {
+            const float alpha = need ? fast_exp2(m_used - mxs) : 1.0f;   // 0 when nothing was kept so far
+            if (need) m_used = mxs;
+            lsum.x *= alpha;
+            lsum.y *= alpha;
+            if (it > 0) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint32_t o[32];
+                    tc_ld32(tO + q * 32, o);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                    tc_st32(tO + q * 32, o);
+                }
+            }
+        }
+        const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+        const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(neg_m, neg_m);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            uint32_t p[32];
+            float2 acc2 = make_float2(0.f, 0.f);
+#pragma unroll
+            for (int qq = 0; qq < 2; ++qq)
+#pragma unroll
+                for (int e = 0; e < 16; ++e) {
+                    float2 x = ffma2(make_float2(__uint_as_float(sr[2 * half + qq][2 * e]),
+                                                 __uint_as_float(sr[2 * half + qq][2 * e + 1])), sc2, nm2);
+                    x.x = fast_exp2(x.x);
+                    x.y = fast_exp2(x.y);
+                    if (qq == 0) lsum = fadd2(lsum, x); else acc2 = fadd2(acc2, x);
+                    p[16 * qq + e] = pack_bf16(x.x, x.y);
+                }
+            lsum = fadd2(lsum, acc2);
+            tc_st32(tS + half * 32, p);                  // P columns [32 half, 32 half + 32) = keys [64 half, 64 half + 64)
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(c.bar(BAR_P_FULL + 2 * t + half));
+        }
+    }
+    if (!c.wait(BAR_O_FULL + t, 0)) return;
+    tc_fence_after();
+    const float inv = 1.0f / (lsum.x + lsum.y);
+    const bool valid = row < c.q_end;
+    __nv_bfloat16 *dst = a.out + ((size_t)(valid ? row - a.q_start : 0) * a.Hq + (c.h0 + t)) * kHeadDim;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint32_t o[32];
+        tc_ld32(tO + q * 32, o);
+        tc_wait_ld();
+        if (valid) {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                uint4 w;
+                w.x = pack_bf16(__uint_as_float(o[8 * e + 0]) * inv, __uint_as_float(o[8 * e + 1]) * inv);
+                w.y = pack_bf16(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv);
+                w.z = pack_bf16(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv);
+                w.w = pack_bf16(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv);
+                *reinterpret_cast<uint4 *>(dst + q * 32 + e * 8) = w;
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, TcArgs a)
 {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t sb = (raw + 1023u) & ~1023u;          // shared-window address of the aligned base
-    unsigned char *sm = smem_raw + (sb - raw);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(sm + OFF_ABORT);
+    Cta c;
+    c.sb = (raw + 1023u) & ~1023u;
+    unsigned char *sm = smem_raw + (c.sb - raw);
+    c.abort_flag = reinterpret_cast<volatile int *>(sm + OFF_ABORT);
+    c.status = a.status;
+    c.bar0 = c.sb + OFF_BAR;
     volatile uint32_t *tmem_ptr_smem = reinterpret_cast<volatile uint32_t *>(sm + OFF_TMEM_PTR);
-    const uint32_t bar0 = sb + OFF_BAR;
-    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
     // a CTA that starts after a wait has run out anywhere does nothing
-    if (tid == 0) *abort_flag = (*reinterpret_cast<volatile uint32_t *>(a.status) & FLUX_STATUS_WAIT_EXPIRED) ? 1 : 0;
+    if (tid == 0) *c.abort_flag = (*reinterpret_cast<volatile uint32_t *>(a.status) & FLUX_STATUS_WAIT_EXPIRED) ? 1 : 0;
     __syncthreads();
-    if (*abort_flag) return;
+    if (*c.abort_flag) return;
 
     // ---- which work item ----
     const int bid = blockIdx.x;
-    const int qt = a.n_qt - 1 - bid / a.n_pairs;          // latest (heaviest) query tiles first
+    c.qt = a.n_qt - 1 - bid / a.n_pairs;                  // latest (heaviest) query tiles first
     const int pr = bid % a.n_pairs;
-    const int kvh = pr / a.ppg, pi = pr % a.ppg;
-    const int h0 = kvh * a.G + 2 * pi;
-    const int nslots = (2 * pi + 1 < a.G) ? 2 : 1;
-    const int q_end = a.q_start + a.Nq;                   // KV rows present
-    const int i0 = a.q_start + qt * BM;
-    const int i_hi = min(i0 + BM - 1, q_end - 1);
+    c.kvh = pr / a.ppg;
+    const int pi = pr % a.ppg;
+    c.h0 = c.kvh * a.G + 2 * pi;
+    c.nslots = (2 * pi + 1 < a.G) ? 2 : 1;
+    c.q_end = a.q_start + a.Nq;                           // KV rows present
+    c.i0 = a.q_start + c.qt * BM;
+    const int i_hi = min(c.i0 + BM - 1, c.q_end - 1);
 
     const uint8_t mode_raw = a.mask[a.req * a.L + a.layer];
     if (mode_raw > 1 && tid == 0) atomicOr(a.status, FLUX_STATUS_BAD_MASK);
-    const bool fa = mode_raw != 0;
-    const int S = a.S, W = a.W;
+    c.fa = mode_raw != 0;
 
     if (bid == 0 && tid == 0) {
-        const int n = q_end;
-        const bool two = !fa && n > S + W;
+        const int n = c.q_end;
+        const bool two = !c.fa && n > a.S + a.W;
         int32_t *d = a.debug;
-        d[0] = fa ? 1 : 0; d[1] = a.layer; d[2] = a.req; d[3] = n;
-        d[4] = 0; d[5] = two ? S : n; d[6] = two ? n - W : 0; d[7] = two ? n : 0;
+        d[0] = c.fa ? 1 : 0; d[1] = a.layer; d[2] = a.req; d[3] = n;
+        d[4] = 0; d[5] = two ? a.S : n; d[6] = two ? n - a.W : 0; d[7] = two ? n : 0;
     }
 
-    int e1, b2;
     const int e2 = i_hi / BN + 1;
-    if (fa) {
-        e1 = 0;
-        b2 = 0;
+    if (c.fa) {
+        c.e1 = 0;
+        c.b2 = 0;
     } else {
-        e1 = min((S + BN - 1) / BN, e2);
-        b2 = max(e1, max(0, i0 - W + 1) / BN);
+        c.e1 = min((a.S + BN - 1) / BN, e2);
+        c.b2 = max(c.e1, max(0, c.i0 - a.W + 1) / BN);
     }
-    const int n_tiles = e1 + max(0, e2 - b2);
+    c.n_tiles = c.e1 + max(0, e2 - c.b2);
 
     // ---- set-up: barriers, TMEM ----
     if (tid == 0) {
-        mbar_init(bar(BAR_Q_FULL), 1);
+        mbar_init(c.bar(BAR_Q_FULL), 1);
         for (int s = 0; s < kKvSlots; ++s) {
-            mbar_init(bar(BAR_KV_FULL + s), 1);
-            mbar_init(bar(BAR_KV_EMPTY + s), 1);
+            mbar_init(c.bar(BAR_KV_FULL + s), 1);
+            mbar_init(c.bar(BAR_KV_EMPTY + s), 1);
         }
         for (int t = 0; t < 2; ++t) {
-            mbar_init(bar(BAR_S_FULL + t), 1);
-            mbar_init(bar(BAR_P_FULL + t), kSoftmaxThreads);
-            mbar_init(bar(BAR_O_FULL + t), 1);
+            mbar_init(c.bar(BAR_S_FULL + t), 1);
+            mbar_init(c.bar(BAR_P_FULL + 2 * t), 4);       // one elected lane per softmax warp
+            mbar_init(c.bar(BAR_P_FULL + 2 * t + 1), 4);
+            mbar_init(c.bar(BAR_O_FULL + t), 1);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 9) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(sb + OFF_TMEM_PTR), "r"(kTmemCols) : "memory");
+                     ::"r"(c.sb + OFF_TMEM_PTR), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem = *tmem_ptr_smem;
+    c.tmem = *tmem_ptr_smem;
 
+    // Each warpgroup executes one setmaxnreg, all four of its warps the same one.
     if (warp >= 8) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
-    if (warp == 8) {
-        // ================= TMA producer =================
-        if (lane == 0) {
-            mbar_expect_tx(bar(BAR_Q_FULL), (uint32_t)(nslots * kTileBytes));
-            for (int t = 0; t < nslots; ++t) {
-                tma_load_3d(sb + OFF_Q + t * kTileBytes, &tm_q, bar(BAR_Q_FULL), 0, h0 + t, qt * BM);
-                tma_load_3d(sb + OFF_Q + t * kTileBytes + kHalfBytes, &tm_q, bar(BAR_Q_FULL), 64, h0 + t, qt * BM);
-            }
-            bool ok = true;
-            for (int it = 0; it < n_tiles && ok; ++it) {
-                const int j0 = tile_of(it, e1, b2) * BN;
-#pragma unroll
-                for (int kv = 0; kv < 2; ++kv) {
-                    const int qi = 2 * it + kv, slot = qi & (kKvSlots - 1), use = qi / kKvSlots;
-                    ok = mbar_wait(bar(BAR_KV_EMPTY + slot), (uint32_t)((use & 1) ^ 1), abort_flag, a.status);
-                    if (!ok) break;
-                    const uint32_t dst = sb + OFF_KV + slot * kTileBytes;
-                    const CUtensorMap *tm = kv ? &tm_v : &tm_k;
-                    mbar_expect_tx(bar(BAR_KV_FULL + slot), (uint32_t)kTileBytes);
-                    tma_load_3d(dst, tm, bar(BAR_KV_FULL + slot), 0, kvh, j0);
-                    tma_load_3d(dst + kHalfBytes, tm, bar(BAR_KV_FULL + slot), 64, kvh, j0);
-                }
-            }
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
+        if (warp == 8) {
+            role_load(c, &tm_q, &tm_k, &tm_v);
+        } else if (warp == 9) {
+            role_mma(c);
         }
-        __syncwarp();
-    } else if (warp == 9) {
-        // ================= MMA issuer =================
-        if (lane == 0) {
-            auto qk = [&](int t, int slot) {   // S_t = Q_t K^T
-                const uint32_t qb = sb + OFF_Q + t * kTileBytes, kb = sb + OFF_KV + slot * kTileBytes;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const uint32_t off = (uint32_t)((kk >> 2) * kHalfBytes + (kk & 3) * 32);
-                    tc_mma_ss(tmem + TM_S + t * 128, smem_desc(qb + off, 16), smem_desc(kb + off, 16), kIdescQK,
-                              kk > 0 ? 1u : 0u);
-                }
-            };
-            auto pv = [&](int t, int slot, bool acc) {   // O_t (+)= P_t V
-                const uint32_t vb = sb + OFF_KV + slot * kTileBytes;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    tc_mma_ts(tmem + TM_O + t * 128, tmem + TM_S + t * 128 + kk * 8,
-                              smem_desc(vb + kk * 2048, kHalfBytes), kIdescPV, (acc || kk > 0) ? 1u : 0u);
-            };
-            bool ok = mbar_wait(bar(BAR_Q_FULL), 0, abort_flag, a.status);
-            if (ok) ok = mbar_wait(bar(BAR_KV_FULL + 0), 0, abort_flag, a.status);
-            if (ok) {
-                tc_fence_after();
-                for (int t = 0; t < nslots; ++t) {
-                    qk(t, 0);
-                    tc_commit(bar(BAR_S_FULL + t));
-                }
-                tc_commit(bar(BAR_KV_EMPTY + 0));
-            }
-            for (int it = 0; it < n_tiles && ok; ++it) {
-                const int vq = 2 * it + 1, vslot = vq & (kKvSlots - 1), vpar = (vq / kKvSlots) & 1;
-                const int kq = 2 * it + 2, kslot = kq & (kKvSlots - 1), kpar = (kq / kKvSlots) & 1;
-                const bool more = it + 1 < n_tiles;
-                ok = mbar_wait(bar(BAR_KV_FULL + vslot), (uint32_t)vpar, abort_flag, a.status);
-                for (int t = 0; t < nslots && ok; ++t) {
-                    ok = mbar_wait(bar(BAR_P_FULL + t), (uint32_t)(it & 1), abort_flag, a.status);
-                    if (!ok) break;
-                    tc_fence_after();
-                    pv(t, vslot, it > 0);
-                    if (t == nslots - 1) tc_commit(bar(BAR_KV_EMPTY + vslot));
-                    if (more) {
-                        if (t == 0) {
-                            ok = mbar_wait(bar(BAR_KV_FULL + kslot), (uint32_t)kpar, abort_flag, a.status);
-                            if (!ok) break;
-                            tc_fence_after();
-                        }
-                        qk(t, kslot);
-                        tc_commit(bar(BAR_S_FULL + t));
-                        if (t == nslots - 1) tc_commit(bar(BAR_KV_EMPTY + kslot));
-                    } else {
-                        tc_commit(bar(BAR_O_FULL + t));
-                    }
-                }
-            }
-        }
-        __syncwarp();
-    }
     } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
-    if (warp < 4 * nslots) {   // (the softmax warps of an unused tile fall through)
-        // ================= softmax of query tile t =================
-        const int t = warp >> 2;
-        const int r = tid & 127;                         // row of the tile = TMEM lane
-        const int row = i0 + r;                          // absolute position of this query
-        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + lane_base + TM_S + t * 128;
-        const uint32_t tO = tmem + lane_base + TM_O + t * 128;
-        float m_used = -INFINITY;                        // running maximum in use, scaled log2 units
-        float l = 0.f;
-        bool ok = true;
-        for (int it = 0; it < n_tiles; ++it) {
-            ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_S_FULL + t), (uint32_t)(it & 1), abort_flag, a.status));
-            if (!ok) break;
-            tc_fence_after();
-            uint32_t sr[4][32];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tc_ld32(tS + c * 32, sr[c]);
-            tc_wait_ld();
-            const int j0 = tile_of(it, e1, b2) * BN;
-            const int jmax = j0 + BN - 1;
-            const bool full = (jmax <= i0) && (fa || jmax < S || j0 > i0 + BM - 1 - W);
-            if (!full) {
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const int key = j0 + c * 32 + e;
-                        const bool keep = key <= row && (fa || key < S || key > row - W);
-                        if (!keep) sr[c][e] = 0xff800000u;   // -inf
-                    }
-            }
-            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-#pragma unroll
-            for (int e = 0; e < 32; ++e) {
-                mx0 = fmaxf(mx0, __uint_as_float(sr[0][e]));
-                mx1 = fmaxf(mx1, __uint_as_float(sr[1][e]));
-                mx2 = fmaxf(mx2, __uint_as_float(sr[2][e]));
-                mx3 = fmaxf(mx3, __uint_as_float(sr[3][e]));
-            }
-            const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * a.scale_log2;
-            const bool need = mx > m_used + kRescaleThreshold;
-            if (__any_sync(0xffffffffu, need)) {
-                const float alpha = need ? fast_exp2(m_used - mx) : 1.0f;   // 0 when nothing was kept so far
-                if (need) m_used = mx;
-                l *= alpha;
-                if (it > 0) {
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        uint32_t o[32];
-                        tc_ld32(tO + c * 32, o);
-                        tc_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                        tc_st32(tO + c * 32, o);
-                    }
-                }
-            }
-            const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-            float l0 = 0.f, l1 = 0.f, l2 = 0.f, l3 = 0.f;
-#pragma unroll
-            for (int c = 0; c < 2; ++c) {
-                uint32_t p[32];
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    const float a0 = fast_exp2(fmaf(__uint_as_float(sr[2 * c][2 * e]), a.scale_log2, neg_m));
-                    const float a1 = fast_exp2(fmaf(__uint_as_float(sr[2 * c][2 * e + 1]), a.scale_log2, neg_m));
-                    const float b0 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1][2 * e]), a.scale_log2, neg_m));
-                    const float b1 = fast_exp2(fmaf(__uint_as_float(sr[2 * c + 1][2 * e + 1]), a.scale_log2, neg_m));
-                    l0 += a0; l1 += a1; l2 += b0; l3 += b1;
-                    p[e] = pack_bf16(a0, a1);
-                    p[16 + e] = pack_bf16(b0, b1);
-                }
-                tc_st32(tS + c * 32, p);                 // P columns [32c, 32c+32) = keys [64c, 64c+64)
-            }
-            l += (l0 + l1) + (l2 + l3);
-            tc_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar(BAR_P_FULL + t));
-        }
-        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(bar(BAR_O_FULL + t), 0, abort_flag, a.status));
-        if (ok) {
-            tc_fence_after();
-            const float inv = 1.0f / l;
-            const bool valid = row < q_end;
-            __nv_bfloat16 *dst = a.out + ((size_t)(valid ? row - a.q_start : 0) * a.Hq + (h0 + t)) * kHeadDim;
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t o[32];
-                tc_ld32(tO + c * 32, o);
-                tc_wait_ld();
-                if (valid) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        uint4 w;
-                        w.x = pack_bf16(__uint_as_float(o[8 * e + 0]) * inv, __uint_as_float(o[8 * e + 1]) * inv);
-                        w.y = pack_bf16(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv);
-                        w.z = pack_bf16(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv);
-                        w.w = pack_bf16(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv);
-                        *reinterpret_cast<uint4 *>(dst + c * 32 + e * 8) = w;
-                    }
-                }
-            }
-        }
-    }
-
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
+        if (warp < 4 * c.nslots) role_softmax(c, a, warp >> 2, warp, lane);
     }
 
     // ---- teardown ----
     tc_fence_before();
     __syncthreads();
-    if (*abort_flag) {
+    if (*c.abort_flag) {
         // let copies and MMAs that were already issued land before the shared memory and TMEM go away
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
     }
     if (warp == 9) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(c.tmem), "r"(kTmemCols) : "memory");
     }
 }
 
