@@ -35,7 +35,7 @@ namespace {
 constexpr int BM = 128, BN = 128;
 constexpr int kHalfBytes = BM * 128;              // 128 rows x 64 bf16 (one 128-byte swizzle span per row)
 constexpr int kTileBytes = 2 * kHalfBytes;        // a 128 x 128 bf16 tile = two halves (d 0-63 | d 64-127)
-constexpr int kKvSlots = 4;
+constexpr int kKvSlots = 5;                        // K and V tiles in flight (ring of 32 KB slots)
 constexpr int kThreads = 384;
 constexpr int kSoftmaxThreads = 128;
 constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // per-thread register targets after rebalancing
@@ -43,9 +43,11 @@ constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // per-thread register targ
 constexpr int OFF_Q = 0;                          // Q tile 0, Q tile 1
 constexpr int OFF_KV = 2 * kTileBytes;
 constexpr int OFF_BAR = OFF_KV + kKvSlots * kTileBytes;
-// mbarriers: Q_FULL | KV_FULL[4] | KV_EMPTY[4] | S_FULL[2] | P_FULL[tile][half] | O_FULL[2]
-constexpr int BAR_Q_FULL = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = 5, BAR_S_FULL = 9, BAR_P_FULL = 11,
-              BAR_O_FULL = 15;
+// mbarriers: Q_FULL | KV_FULL[slots] | KV_EMPTY[slots] | S_FULL[2] | P_FULL[tile][half] | O_FULL[2]
+constexpr int BAR_Q_FULL = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = BAR_KV_FULL + kKvSlots,
+              BAR_S_FULL = BAR_KV_EMPTY + kKvSlots, BAR_P_FULL = BAR_S_FULL + 2, BAR_O_FULL = BAR_P_FULL + 4,
+              kNumBars = BAR_O_FULL + 2;
+static_assert(kNumBars <= 24, "barrier area");
 constexpr int OFF_TMEM_PTR = OFF_BAR + 24 * 8;
 constexpr int OFF_ABORT = OFF_TMEM_PTR + 4;
 constexpr int kSmemBytes = OFF_BAR + 256 + 1024;  // + slack to align the base to 1024 bytes
@@ -263,7 +265,7 @@ __device__ __forceinline__ void role_load(const Cta &c, const CUtensorMap *tm_q,
         const int j0 = tile_of(it, c.e1, c.b2) * BN;
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
-            const int qi = 2 * it + kv, slot = qi & (kKvSlots - 1), use = qi / kKvSlots;
+            const int qi = 2 * it + kv, slot = qi % kKvSlots, use = qi / kKvSlots;
             if (!c.wait(BAR_KV_EMPTY + slot, (uint32_t)((use & 1) ^ 1))) return;
             const uint32_t dst = c.sb + OFF_KV + slot * kTileBytes;
             const CUtensorMap *tm = kv ? tm_v : tm_k;
@@ -278,7 +280,8 @@ __device__ __forceinline__ void role_load(const Cta &c, const CUtensorMap *tm_q,
 
 // ================= MMA issuer (one warp, one issuing lane) =================
 // Issue order per KV tile j:  PV_0[j] QK_0[j+1] PV_1[j] QK_1[j+1]; the tensor pipe runs them in
-// that order, so S_t[j+1] overwrites S_t / P_t only after PV_t[j] has read P_t[j].
+// that order, so S_t[j+1] overwrites S_t / P_t only after PV_t[j] has read P_t[j].  (One issuer for
+// both tiles: two issuing warps, whose MMAs interleave instruction by instruction, ran slower.)
 __device__ __forceinline__ void role_mma(const Cta &c)
 {
     // S_t = Q_t K^T, then up to two commits (tcgen05.commit belongs to the issuing lane; 0 = none)
@@ -315,8 +318,8 @@ __device__ __forceinline__ void role_mma(const Cta &c)
     for (int t = 0; t < c.nslots; ++t)
         qk(t, 0, c.bar(BAR_S_FULL + t), t == c.nslots - 1 ? c.bar(BAR_KV_EMPTY + 0) : 0u);
     for (int it = 0; it < c.n_tiles; ++it) {
-        const int vq = 2 * it + 1, vslot = vq & (kKvSlots - 1), vpar = (vq / kKvSlots) & 1;
-        const int kq = 2 * it + 2, kslot = kq & (kKvSlots - 1), kpar = (kq / kKvSlots) & 1;
+        const int vq = 2 * it + 1, vslot = vq % kKvSlots, vpar = (vq / kKvSlots) & 1;
+        const int kq = 2 * it + 2, kslot = kq % kKvSlots, kpar = (kq / kKvSlots) & 1;
         const bool more = it + 1 < c.n_tiles;
         if (!c.wait(BAR_KV_FULL + vslot, (uint32_t)vpar)) return;
         for (int t = 0; t < c.nslots; ++t) {
