@@ -227,6 +227,13 @@ int flux_profile_read(flux_plan *plan, int32_t kind, double *total_ms, int64_t *
 #define FLUX_PREFILL_TCGEN05  2
 int flux_debug_prefill_kernel(flux_plan *plan, int32_t which);
 
+/* Exercises the give-up path of the kernels' bounded waits without any fault: launches one warp
+ * that waits, with the same bounded wait the prefill kernel uses, on a barrier nothing arrives
+ * at.  After limit_cycles SM clock cycles (1 .. 2e9) the wait runs out, the kernel sets
+ * FLUX_STATUS_WAIT_EXPIRED and returns; flux_plan_status() then reports FLUX_E_DEVICE_TIMEOUT
+ * and clears the word.  While the bit is set, prefill CTAs return at once without computing. */
+int flux_debug_wait_probe(flux_plan *plan, int64_t limit_cycles, void *stream);
+
 /* Number of kernels this plan has launched so far (host counter). */
 int64_t flux_launch_count(const flux_plan *plan);
 

@@ -419,6 +419,15 @@ int flux_attn_prefill(flux_plan *plan, int32_t layer, int32_t req, const void *q
     return launch_prefill(plan, layer, req, q, k, v, q_start, Nq, out, (cudaStream_t)stream);
 }
 
+int flux_debug_wait_probe(flux_plan *plan, int64_t limit_cycles, void *stream)
+{
+    int rc = need_plan(plan, true);
+    if (rc) return rc;
+    if (limit_cycles < 1 || limit_cycles > 2000000000ll)
+        return fail(FLUX_E_INVALID_ARG, "limit_cycles must be in [1, 2e9]");
+    return launch_wait_probe(plan, limit_cycles, (cudaStream_t)stream);
+}
+
 int flux_debug_prefill_kernel(flux_plan *plan, int32_t which)
 {
     int rc = need_plan(plan, false);

@@ -99,7 +99,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
 }
 // Bounded wait: false when the CTA is aborting or the limit ran out (which raises the flag).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
-                                          uint32_t *status)
+                                          uint32_t *status, long long limit = kWaitCycles)
 {
     if (mbar_try(bar, parity)) return true;
     const long long t0 = clock64();
@@ -108,7 +108,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         for (int i = 0; i < 64; ++i)
             if (mbar_try(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitCycles) {
+        if (clock64() - t0 > limit) {
             *abort_flag = 1;
             atomicOr(status, FLUX_STATUS_WAIT_EXPIRED);
             return false;
@@ -555,6 +555,23 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     }
 }
 
+// One warp waits, with the bounded wait the prefill kernel uses, on an mbarrier nothing ever
+// arrives at: the wait runs out after `limit` cycles, raises FLUX_STATUS_WAIT_EXPIRED and the
+// kernel returns normally.  Exists so that the give-up path can be exercised without a fault.
+__global__ void wait_probe_kernel(uint32_t *status, long long limit)
+{
+    __shared__ __align__(8) unsigned long long bar_storage;
+    __shared__ int abort_flag;
+    const uint32_t bar = smem_u32(&bar_storage);
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    mbar_wait(bar, 0, &abort_flag, status, limit);
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -598,6 +615,13 @@ int prefill_tc_setup()
                     fa.numRegs);
     return check_cuda(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes),
                       "cudaFuncSetAttribute(prefill_tc_kernel)");
+}
+
+int launch_wait_probe(flux_plan *p, long long limit_cycles, cudaStream_t st)
+{
+    wait_probe_kernel<<<1, 32, 0, st>>>((uint32_t *)((char *)p->ws + p->lay.status), limit_cycles);
+    p->launches++;
+    return check_cuda(cudaGetLastError(), "wait probe launch");
 }
 
 int launch_prefill_tc(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v, int q_start,

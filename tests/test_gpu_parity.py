@@ -152,6 +152,28 @@ def test_prefill_small_shapes(flux, N, Hq, Hkv, S, W, chunks, kernel):
     assert plan.flux_plan_status() == 0
 
 
+@pytest.mark.parametrize("kernel", [2, 1], ids=["tcgen05", "warp_mma"])
+def test_prefill_scores_rising_along_the_sequence(flux, kernel):
+    """Keys whose scores grow by tens of log2 units from one KV tile to the next, so the running
+    maximum has to be raised (and the accumulator rescaled) again and again in the middle of a row;
+    and the mirror case, where the first keys dominate and later tiles underflow to nothing."""
+    N, Hq, Hkv, S, W = 1100, 4, 2, 64, 300
+    plan = _plan(flux, 2, Hq, Hkv, S, W, 1, 2048)
+    plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
+    plan.flux_debug_prefill_kernel(kernel)
+    q = synth.normal_bf16((N, Hq, 128), 4242, 1, DEV).float() + 1.0
+    v = synth.normal_bf16((N, Hkv, 128), 4242, 3, DEV)
+    ramp = torch.linspace(0.0, 3.0, N, device=DEV)[:, None, None]
+    for sign in (1.0, -1.0):
+        k = (synth.normal_bf16((N, Hkv, 128), 4242, 2, DEV).float() + sign * ramp).to(torch.bfloat16)
+        qb = q.to(torch.bfloat16)
+        for layer, mode in ((0, oracle.FA), (1, oracle.SA)):
+            out = plan.flux_attn_prefill(layer, 0, qb, k, v, 0)
+            ref = oracle.prefill(mode, bits(qb), bits(k), bits(v), 0, S, W, _scale())
+            compare(out, ref, "rising scores sign=%+.0f mode=%d" % (sign, mode))
+    assert plan.flux_plan_status() == 0
+
+
 DECODE_CASES = [
     # Hq, Hkv, S, W, context lengths (0 = inactive request), layout
     (8, 2, 4, 8, [1, 12, 13, 40], 0),
@@ -234,6 +256,28 @@ def test_router_inputs_and_device_flags(flux):
         plan.flux_router_apply(mask=np.array([[1, 0, 2]], dtype=np.uint8))
     plan.flux_router_apply(mask=torch.tensor([[1, 0, 2]], dtype=torch.uint8, device=DEV))
     assert plan.flux_plan_status(raise_on_flag=False) == flux.FLUX_STATUS_BAD_MASK
+
+
+def test_bounded_wait_gives_up_and_reports(flux):
+    """A device-side wait that nothing satisfies runs out after its limit, sets the status bit and
+    the kernel returns; the context stays usable and the next prefill is correct again."""
+    plan = _plan(flux, 1, 4, 2, 8, 16, 1, 256)
+    plan.flux_router_apply(mask=np.array([[1]], dtype=np.uint8))
+    q = synth.normal_bf16((200, 4, 128), 31, 1, DEV)
+    k = synth.normal_bf16((200, 2, 128), 31, 2, DEV)
+    v = synth.normal_bf16((200, 2, 128), 31, 3, DEV)
+    ref = oracle.prefill(oracle.FA, bits(q), bits(k), bits(v), 0, 8, 16, _scale())
+    plan.flux_debug_wait_probe(2_000_000)                      # about a millisecond
+    with pytest.raises(flux.FluxError) as e:
+        plan.flux_plan_status()
+    assert e.value.code == flux.FLUX_E_DEVICE_TIMEOUT
+    assert plan.flux_plan_status() == 0                        # reading cleared the word
+    plan.flux_debug_wait_probe(2_000_000)
+    out = plan.flux_attn_prefill(0, 0, q, k, v, 0, torch.zeros_like(q))   # CTAs see the bit and do nothing
+    assert plan.flux_plan_status(raise_on_flag=False) == flux.FLUX_STATUS_WAIT_EXPIRED
+    assert torch.count_nonzero(out) == 0
+    compare(plan.flux_attn_prefill(0, 0, q, k, v, 0), ref, "prefill after a timed-out wait")
+    assert plan.flux_plan_status() == 0
 
 
 def test_host_side_argument_errors_launch_nothing(flux):
