@@ -55,6 +55,11 @@ def lib():
         L.flux_oracle_prefill_rows.argtypes = [ctypes.c_int, vp, vp, vp, i64, i64, vp, vp, i64,
                                                ctypes.c_int, ctypes.c_int, ctypes.c_int, i64, i64,
                                                dbl, vp]
+        L.flux_oracle_kept_blocks.restype = i64
+        L.flux_oracle_kept_blocks.argtypes = [i64, i64, vp, i64, vp]
+        L.flux_oracle_prefill_blocks.restype = None
+        L.flux_oracle_prefill_blocks.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, i64, ctypes.c_int,
+                                                 ctypes.c_int, ctypes.c_int, i64, vp, i64, dbl, vp]
         L.flux_oracle_decode.restype = None
         L.flux_oracle_decode.argtypes = [ctypes.c_int, vp, vp, vp, i64, i64, ctypes.c_int,
                                          ctypes.c_int, ctypes.c_int, i64, i64, dbl, vp,
@@ -164,6 +169,49 @@ def prefill_rows(mode, Q, K, V, q_start, rows, heads, S, W, scale):
     O = np.empty((len(rows), D), dtype=np.float64)
     lib().flux_oracle_prefill_rows(mode, _p(Q), _p(K), _p(V), _kv_stride(K), q_start, _p(rows),
                                    _p(heads), len(rows), Hq, Hkv, D, S, W, float(scale), _p(O))
+    return O
+
+
+def kept_blocks(i: int, B: int, bm: np.ndarray) -> np.ndarray:
+    """Sorted key positions query position ``i`` attends to under the block mask ``bm[qb][kb]``
+    (block size ``B``; causal inside kept blocks)."""
+    bm = np.ascontiguousarray(bm, dtype=np.uint8)
+    assert bm.ndim == 2 and i // B < bm.shape[0] and i // B < bm.shape[1]
+    idx = np.empty(i + 1, dtype=np.int64)
+    n = lib().flux_oracle_kept_blocks(int(i), int(B), _p(bm), bm.shape[1], _p(idx))
+    return idx[:n].copy()
+
+
+def streaming_block_mask(n_qb: int, n_kb: int, S: int, W: int, B: int) -> np.ndarray:
+    """The streaming pattern (sink + local window, Table 3) at block granularity: query block qb
+    keeps the key blocks that hold sink positions and the ceil(W / B) blocks ending with its own."""
+    qb = np.arange(n_qb)[:, None]
+    kb = np.arange(n_kb)[None, :]
+    n_sink = -(-S // B)
+    n_local = -(-W // B)
+    return ((kb <= qb) & ((kb < n_sink) | (kb > qb - n_local))).astype(np.uint8)
+
+
+def prefill_blocks(Q, K, V, q_start, B, bm, scale, rows=None, heads=None):
+    """Prefill under a block mask.  ``rows`` / ``heads`` (equal-length arrays of absolute query
+    positions and query heads) select outputs -> ``[n][D]``; otherwise ``[Nq][Hq][D]``."""
+    Q = np.ascontiguousarray(Q)
+    Nq, Hq, D = Q.shape
+    Hkv = K.shape[1]
+    bm = np.ascontiguousarray(bm, dtype=np.uint8)
+    assert K.shape[0] >= q_start + Nq and V.shape == K.shape and V.strides == K.strides
+    assert bm.shape[0] * B >= q_start + Nq and bm.shape[1] * B >= q_start + Nq
+    if rows is None:
+        O = np.empty((Nq, Hq, D), dtype=np.float64)
+        lib().flux_oracle_prefill_blocks(_p(Q), _p(K), _p(V), _kv_stride(K), q_start, Nq, None, None, 0, Hq,
+                                         Hkv, D, int(B), _p(bm), bm.shape[1], float(scale), _p(O))
+        return O
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    heads = np.ascontiguousarray(heads, dtype=np.int32)
+    assert len(rows) == len(heads) and rows.min() >= q_start and rows.max() < q_start + Nq
+    O = np.empty((len(rows), D), dtype=np.float64)
+    lib().flux_oracle_prefill_blocks(_p(Q), _p(K), _p(V), _kv_stride(K), q_start, Nq, _p(rows), _p(heads),
+                                     len(rows), Hq, Hkv, D, int(B), _p(bm), bm.shape[1], float(scale), _p(O))
     return O
 
 

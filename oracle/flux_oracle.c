@@ -158,6 +158,63 @@ void flux_oracle_prefill_rows(int mode, const uint16_t *Q, const uint16_t *K,
     }
 }
 
+/* ---- block-granular sparse patterns ----------------------------------------
+ * The sparse kernels the paper runs select keys in blocks (Appendix D.3: the
+ * block size, 64, is "the minimum unit of sparsity"; Sec. 4.1 lists block
+ * patterns -- streaming, XAttention's selected blocks -- as the sparse modes).
+ * A block mask bm[qb][kb] (row-major, n_kb entries per row) says whether query
+ * block qb (positions [qb*B, (qb+1)*B)) attends to key block kb; inside a kept
+ * block causality still holds:
+ *     kept(i) = { j : 0 <= j <= i  and  bm[i / B][j / B] != 0 }
+ * B = 1 makes bm an arbitrary token-level mask.  Writes the sorted list into
+ * idx (room for i+1 entries, may be NULL) and returns its size. */
+int64_t flux_oracle_kept_blocks(int64_t i, int64_t B, const uint8_t *bm,
+                                int64_t n_kb, int64_t *idx)
+{
+    int64_t cnt = 0;
+    const uint8_t *row = bm + (i / B) * n_kb;
+    for (int64_t j = 0; j <= i; ++j) {
+        if (row[j / B] != 0) {
+            if (idx) idx[cnt] = j;
+            ++cnt;
+        }
+    }
+    return cnt;
+}
+
+/* Prefill rows under a block mask (Eq. 2 with the condensed subset given by the
+ * mask).  rows / heads as in flux_oracle_prefill_rows; rows == NULL evaluates
+ * every (row, head) of the chunk in order, O then [Nq][Hq][D].  A query whose
+ * kept set is empty gets a zero row. */
+void flux_oracle_prefill_blocks(const uint16_t *Q, const uint16_t *K,
+                                const uint16_t *V, int64_t kv_tok_stride,
+                                int64_t q_start, int64_t Nq, const int64_t *rows,
+                                const int32_t *heads, int64_t n_rows, int Hq,
+                                int Hkv, int D, int64_t B, const uint8_t *bm,
+                                int64_t n_kb, double scale, double *O)
+{
+    int G = Hq / Hkv;
+    int64_t total = rows ? n_rows : Nq * Hq;
+#pragma omp parallel for schedule(dynamic, 4)
+    for (int64_t t = 0; t < total; ++t) {
+        int64_t i = rows ? rows[t] : q_start + t / Hq;
+        int h = rows ? heads[t] : (int)(t % Hq);
+        int64_t *idx = (int64_t *)malloc(sizeof(int64_t) * (size_t)(i + 1));
+        int64_t n_idx = flux_oracle_kept_blocks(i, B, bm, n_kb, idx);
+        double *o = O + t * (int64_t)D;
+        if (n_idx == 0) {
+            for (int d = 0; d < D; ++d) o[d] = 0.0;
+        } else {
+            int g = h / G;
+            flux_oracle_attend(Q + ((i - q_start) * Hq + h) * (int64_t)D,
+                               K + (int64_t)g * D, V + (int64_t)g * D,
+                               kv_tok_stride, idx, n_idx, D, scale, o, NULL,
+                               NULL, NULL);
+        }
+        free(idx);
+    }
+}
+
 /* ---- one decode step of one layer for one request --------------------------
  * The new token's K, V were appended first, so the cache holds positions
  * 0 .. n-1 and the query sits at position n-1 (Sec. 3.3).  q, o: [Hq][D].

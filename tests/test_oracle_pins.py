@@ -307,3 +307,66 @@ def test_decode_byte_ratio_matches_paper_speedup():
     assert rows_fa == n and rows_sa == S + W
     ratio = rows_fa / ((1 - omega) * rows_fa + omega * rows_sa)
     assert lo < ratio < hi
+
+
+# ---- block-granular masks ---------------------------------------------------------
+
+_BM_B2 = np.array([[1, 0, 0, 0], [0, 1, 0, 0], [1, 0, 1, 0], [1, 1, 0, 1]], dtype=np.uint8)
+
+
+def test_block_mask_kept_sets_match_hand_enumeration():
+    for _, i, want in _read_sets("kept_blocks_B2.txt"):
+        assert oracle.kept_blocks(i, 2, _BM_B2).tolist() == want, i
+
+
+def test_block_mask_with_unit_blocks_reproduces_sa_and_full_mask_reproduces_fa():
+    """B = 1 turns the block mask into a token mask: fed with the sink + window sets it must give
+    exactly the SA prefill; the lower-triangular mask at B = 4 must give exactly the FA prefill."""
+    rng = np.random.default_rng(21)
+    N, Hq, Hkv, D, S, W = 23, 4, 2, 8, 3, 5
+    Q, K, V = (_rand_bits(rng, s) for s in [(N, Hq, D), (N, Hkv, D), (N, Hkv, D)])
+    tok = np.zeros((N, N), dtype=np.uint8)
+    for i in range(N):
+        tok[i, oracle.kept(oracle.SA, i, S, W)] = 1
+    assert np.array_equal(oracle.prefill_blocks(Q, K, V, 0, 1, tok, 0.3), oracle.prefill(oracle.SA, Q, K, V, 0, S, W, 0.3))
+    nb = -(-N // 4)
+    tri = np.tril(np.ones((nb, nb), dtype=np.uint8))
+    assert np.array_equal(oracle.prefill_blocks(Q, K, V, 0, 4, tri, 0.3), oracle.prefill(oracle.FA, Q, K, V, 0, 0, 1, 0.3))
+    # chunked evaluation and row selection address the same rows
+    full = oracle.prefill_blocks(Q, K, V, 0, 4, tri, 0.3)
+    part = oracle.prefill_blocks(Q[8:], K, V, 8, 4, tri, 0.3)
+    assert np.array_equal(part, full[8:])
+    rows, heads = np.array([0, 9, 22]), np.array([3, 0, 2])
+    assert np.array_equal(oracle.prefill_blocks(Q, K, V, 0, 4, tri, 0.3, rows, heads), full[rows, heads])
+
+
+def test_block_mask_prefill_matches_python_brute_force_and_empty_rows_are_zero():
+    rng = np.random.default_rng(22)
+    N, Hq, Hkv, D = 8, 2, 1, 4
+    Q, K, V = (_rand_bits(rng, s) for s in [(N, Hq, D), (N, Hkv, D), (N, Hkv, D)])
+    Qf, Kf, Vf = (oracle.bits_to_f64(x) for x in (Q, K, V))
+    O = oracle.prefill_blocks(Q, K, V, 0, 2, _BM_B2, 0.7)
+    for _, i, idx in _read_sets("kept_blocks_B2.txt"):
+        for h in range(Hq):
+            assert np.allclose(O[i, h], _brute(Qf, Kf, Vf, i, h, Hq // Hkv, idx, 0.7), rtol=0, atol=1e-13)
+    bm = _BM_B2.copy()
+    bm[1, 1] = 0                                     # query block 1 keeps nothing
+    O2 = oracle.prefill_blocks(Q, K, V, 0, 2, bm, 0.7)
+    assert not O2[2:4].any() and np.array_equal(O2[4:], O[4:])
+
+
+@pytest.mark.parametrize("S,W,B", [(128, 2048, 64), (64, 256, 64), (5, 7, 4), (0, 1, 2), (130, 100, 64)])
+def test_streaming_block_mask_brackets_the_token_exact_sets(S, W, B):
+    """The block-granular streaming mask keeps every position the token-exact sink + window set
+    keeps, and nothing the set with sink and window each widened by B - 1 positions would not keep."""
+    N = max(6 * B, S + W + 2 * B) + 3
+    nb = -(-N // B)
+    bm = oracle.streaming_block_mask(nb, nb, S, W, B)
+    assert bm.shape == (nb, nb) and not np.triu(bm, 1).any() and bm.diagonal().all()
+    for i in list(range(0, min(N, 3 * B + 2))) + [S + W - 1, S + W, S + W + B, N - B - 1, N - 1]:
+        got = set(oracle.kept_blocks(i, B, bm).tolist())
+        lo = set(oracle.kept(oracle.SA, i, S, W).tolist())
+        hi = set(oracle.kept(oracle.SA, i, S + B - 1, W + B - 1).tolist())
+        assert lo <= got <= hi, (i, sorted(got - hi), sorted(lo - got))
+    # a row far from both ends keeps ceil(S/B) sink blocks and ceil(W/B) local blocks
+    assert int(bm[nb - 1].sum()) == min(nb, -(-S // B) + -(-W // B))
