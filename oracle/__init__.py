@@ -184,7 +184,8 @@ def kept_blocks(i: int, B: int, bm: np.ndarray) -> np.ndarray:
 
 def streaming_block_mask(n_qb: int, n_kb: int, S: int, W: int, B: int) -> np.ndarray:
     """The streaming pattern (sink + local window, Table 3) at block granularity: query block qb
-    keeps the key blocks that hold sink positions and the ceil(W / B) blocks ending with its own."""
+    keeps the key blocks that hold sink positions and the ceil(W / B) blocks ending with its own
+    (so a row sees between W - B + 1 and W local positions when B divides W)."""
     qb = np.arange(n_qb)[:, None]
     kb = np.arange(n_kb)[None, :]
     n_sink = -(-S // B)

@@ -357,16 +357,18 @@ def test_block_mask_prefill_matches_python_brute_force_and_empty_rows_are_zero()
 
 @pytest.mark.parametrize("S,W,B", [(128, 2048, 64), (64, 256, 64), (5, 7, 4), (0, 1, 2), (130, 100, 64)])
 def test_streaming_block_mask_brackets_the_token_exact_sets(S, W, B):
-    """The block-granular streaming mask keeps every position the token-exact sink + window set
-    keeps, and nothing the set with sink and window each widened by B - 1 positions would not keep."""
+    """Block granularity can only round: the sink up to whole blocks, the window to the ceil(W / B)
+    blocks that end with the query's own (so a row sees between W' - B + 1 and W' local positions,
+    W' = W rounded up to blocks).  The kept set therefore lies between the two token-exact sets."""
     N = max(6 * B, S + W + 2 * B) + 3
     nb = -(-N // B)
     bm = oracle.streaming_block_mask(nb, nb, S, W, B)
     assert bm.shape == (nb, nb) and not np.triu(bm, 1).any() and bm.diagonal().all()
     for i in list(range(0, min(N, 3 * B + 2))) + [S + W - 1, S + W, S + W + B, N - B - 1, N - 1]:
         got = set(oracle.kept_blocks(i, B, bm).tolist())
-        lo = set(oracle.kept(oracle.SA, i, S, W).tolist())
-        hi = set(oracle.kept(oracle.SA, i, S + B - 1, W + B - 1).tolist())
+        Wb = -(-W // B) * B
+        lo = set(oracle.kept(oracle.SA, i, S, max(1, Wb - B + 1)).tolist())
+        hi = set(oracle.kept(oracle.SA, i, -(-S // B) * B, Wb).tolist())
         assert lo <= got <= hi, (i, sorted(got - hi), sorted(lo - got))
     # a row far from both ends keeps ceil(S/B) sink blocks and ceil(W/B) local blocks
     assert int(bm[nb - 1].sum()) == min(nb, -(-S // B) + -(-W // B))
