@@ -306,6 +306,26 @@ def prefill_block(flux, dev, peaks, warmup):
         "tflops_mix": total_flop / wall_ms / 1e9,
         "gpu_launches": cnt_all,
     }
+    # the same sparse pattern at block granularity (64-position blocks) through the block-mask entry point
+    nb = N // 64
+    qb = np.arange(nb)[:, None]; kb = np.arange(nb)[None, :]
+    bm = ((kb <= qb) & ((kb < -(-S // 64)) | (kb > qb - -(-W // 64)))).astype(np.uint8)
+    bm_dev = torch.from_numpy(bm).to(dev)
+    for _ in range(max(1, warmup)):
+        plan.flux_attn_prefill_blocks(q, k, v, 0, bm_dev, out)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(5):
+        plan.flux_attn_prefill_blocks(q, k, v, 0, bm_dev, out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms_blk = e0.elapsed_time(e1) / 5
+    off = bm.sum(axis=1).astype(np.int64) - 1                     # kept blocks below the diagonal, per query block
+    pairs_blk = int((off * 64 * 64).sum() + nb * (64 * 65 // 2))  # + the causal half of each diagonal block
+    res["block_mask_sa"] = {"kernel": "prefill_blocks_kernel (mma.sync, 64 x 64 blocks)", "pattern":
+                            "streaming at block granularity: %d sink + %d local blocks" % (-(-S // 64), -(-W // 64)),
+                            "ms_layer": ms_blk, "tflops": 4 * Hq * D * pairs_blk / ms_blk / 1e9}
     if ms_fa is not None:
         ach = flop_fa / ms_fa / 1e9
         res["roofline"] = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],

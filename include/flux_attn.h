@@ -112,6 +112,21 @@ int flux_attn_prefill(flux_plan *plan, int32_t layer, int32_t req, const void *q
                       const void *k, const void *v, int32_t q_start, int32_t Nq,
                       void *out, void *stream);
 
+/* Prefill of one request under a block mask: Sparse Attention (Eq. 2) whose condensed key subset
+ * is given in blocks of 64 positions, the unit in which the sparse kernels the paper runs select
+ * keys (Appendix D.3, "block size"; Sec. 4.1 names the block patterns).  Query position i attends
+ * to { j <= i : block_mask[i / 64][j / 64] != 0 }: causality still holds inside a kept block.
+ *   block_mask  uint8 [n_q_blocks][n_kv_blocks], device, row-major; rows are ABSOLUTE query blocks
+ *               (row (q_start + r) / 64 serves chunk row r), so one matrix serves every chunk;
+ *               entries beyond the diagonal are ignored.  n_kv_blocks <= 4096 (else FLUX_E_CAPACITY).
+ *   q, out      [Nq][n_q_heads][head_dim], device; k, v as in flux_attn_prefill.
+ *   q_start     multiple of 64.
+ * Independent of the routing decision (no layer / request arguments).  A query whose mask row
+ * keeps no block up to its own gets a zero output row and raises FLUX_STATUS_BAD_MASK. */
+int flux_attn_prefill_blocks(flux_plan *plan, const void *q, const void *k, const void *v,
+                             int32_t q_start, int32_t Nq, const uint8_t *block_mask,
+                             int32_t n_kv_blocks, void *out, void *stream);
+
 /* Sparse-decode KV retention after prefill (Sec. 3.3: a sparse layer keeps only
  * the rows its kernel needs).  Copies, for one (layer, request), the rows of
  * k_src/v_src ([n][n_kv_heads][head_dim], row = position) that decode will need

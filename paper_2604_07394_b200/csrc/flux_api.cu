@@ -419,6 +419,26 @@ int flux_attn_prefill(flux_plan *plan, int32_t layer, int32_t req, const void *q
     return launch_prefill(plan, layer, req, q, k, v, q_start, Nq, out, (cudaStream_t)stream);
 }
 
+int flux_attn_prefill_blocks(flux_plan *plan, const void *q, const void *k, const void *v, int32_t q_start,
+                             int32_t Nq, const uint8_t *block_mask, int32_t n_kv_blocks, void *out, void *stream)
+{
+    int rc = need_plan(plan, true);
+    if (rc) return rc;
+    if (Nq < 0 || q_start < 0) return fail(FLUX_E_INVALID_ARG, "negative q_start or Nq");
+    if (q_start % 64) return fail(FLUX_E_INVALID_ARG, "q_start must be a multiple of the block size (64)");
+    if ((int64_t)q_start + Nq > plan->cfg.max_context)
+        return fail(FLUX_E_CAPACITY, "q_start + Nq = %lld exceeds max_context %d",
+                    (long long)q_start + Nq, plan->cfg.max_context);
+    if (Nq == 0) return FLUX_OK;
+    if ((int64_t)n_kv_blocks * 64 < (int64_t)q_start + Nq)
+        return fail(FLUX_E_INVALID_ARG, "block mask rows of %d blocks do not cover %lld positions", n_kv_blocks,
+                    (long long)q_start + Nq);
+    if (!q || !k || !v || !out || !block_mask) return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
+        return fail(FLUX_E_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    return launch_prefill_blocks(plan, q, k, v, q_start, Nq, block_mask, n_kv_blocks, out, (cudaStream_t)stream);
+}
+
 int flux_debug_wait_probe(flux_plan *plan, int64_t limit_cycles, void *stream)
 {
     int rc = need_plan(plan, true);

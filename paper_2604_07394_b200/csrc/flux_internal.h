@@ -100,6 +100,8 @@ int launch_prefill(flux_plan *p, int layer, int req, const void *q, const void *
 // bracket a dominant-kernel launch with events when profiling is on
 int prof_begin(flux_plan *p, int kind, cudaStream_t st);   // returns record index or -1
 void prof_end(flux_plan *p, int rec, cudaStream_t st);
+int launch_prefill_blocks(flux_plan *p, const void *q, const void *k, const void *v, int q_start, int Nq,
+                          const uint8_t *block_mask, int n_kv_blocks, void *out, cudaStream_t st);
 int launch_wait_probe(flux_plan *p, long long limit_cycles, cudaStream_t st);
 int decode_setup(flux_plan *p);   // one-time attribute setting for the decode kernel
 int prefill_setup(flux_plan *p);

@@ -7,6 +7,7 @@ int prefill_mma_setup();
 int launch_prefill_mma(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v,
                        int q_start, int Nq, void *out, cudaStream_t st);
 int prefill_tc_setup();
+int prefill_blocks_setup();
 int launch_prefill_tc(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v,
                       int q_start, int Nq, void *out, cudaStream_t st);
 
@@ -15,6 +16,7 @@ int prefill_setup(flux_plan *p)
     p->prefill_kernel = FLUX_PREFILL_AUTO;
     int rc = prefill_mma_setup();
     if (!rc) rc = prefill_tc_setup();
+    if (!rc) rc = prefill_blocks_setup();
     return rc;
 }
 

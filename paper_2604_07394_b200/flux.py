@@ -43,7 +43,7 @@ FLUX_KV_COMPACT_SA = 1
 
 EXPORTS = [
     "flux_plan_create", "flux_plan_destroy", "flux_workspace_size", "flux_plan_set_workspace",
-    "flux_router_apply", "flux_attn_prefill", "flux_kv_retain", "flux_kv_append",
+    "flux_router_apply", "flux_attn_prefill", "flux_attn_prefill_blocks", "flux_kv_retain", "flux_kv_append",
     "flux_attn_decode", "flux_attn_decode_noalloc", "flux_attn_decode_host", "flux_attn_prefill_host", "flux_plan_status",
     "flux_debug_dispatch", "flux_debug_prefill_kernel", "flux_debug_wait_probe", "flux_profile_enable", "flux_profile_read", "flux_launch_count", "flux_last_error", "flux_version",
 ]
@@ -85,6 +85,7 @@ def load():
     L.flux_plan_set_workspace.argtypes = [vp, vp, sz]
     L.flux_router_apply.argtypes = [vp, vp, vp, i32, vp, vp]
     L.flux_attn_prefill.argtypes = [vp, i32, i32, vp, vp, vp, i32, i32, vp, vp]
+    L.flux_attn_prefill_blocks.argtypes = [vp, vp, vp, vp, i32, i32, vp, i32, vp, vp]
     L.flux_kv_retain.argtypes = [vp, i32, i32, vp, vp, i32, vp, vp, vp]
     L.flux_kv_append.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
@@ -190,6 +191,15 @@ class Plan:
             out = torch.empty_like(q)
         _check(load().flux_attn_prefill(self._h, layer, req, _ptr(q), _ptr(k), _ptr(v), q_start, Nq,
                                         _ptr(out), _stream()))
+        return out
+
+    def flux_attn_prefill_blocks(self, q, k, v, q_start, block_mask, out=None):
+        """block_mask: uint8 device tensor [n_q_blocks][n_kv_blocks], rows = absolute query blocks."""
+        Nq = int(q.shape[0])
+        if out is None:
+            out = torch.empty_like(q)
+        _check(load().flux_attn_prefill_blocks(self._h, _ptr(q), _ptr(k), _ptr(v), q_start, Nq,
+                                               _ptr(block_mask), int(block_mask.shape[1]), _ptr(out), _stream()))
         return out
 
     def flux_attn_prefill_host(self, layer, req, q_host, q_dev, k, v, q_start, out_dev, out_host):
