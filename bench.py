@@ -153,9 +153,9 @@ class DecodeBench:
 
     def step(self, t):
         p, w = self.plan, self.w
-        for l in range(w.n_layers):
-            p.flux_kv_append(l, w.batch, self.kn[l], self.vn[l], self.ktab[l], self.vtab[l], self.pos[t])
-            p.flux_attn_decode(l, w.batch, self.q[l], self.ktab[l], self.vtab[l], self.ctx[t], self.out[l])
+        for l in range(w.n_layers):      # append + attend of a layer in one launch, then the combine pass
+            p.flux_attn_decode_step(l, w.batch, self.q[l], self.kn[l], self.vn[l], self.ktab[l], self.vtab[l],
+                                    self.ctx[t], self.out[l])
 
     def capture_step(self, t_next):
         """One decode step (all layers) as a CUDA graph.  The step's positions live in two device
@@ -167,8 +167,8 @@ class DecodeBench:
         self.graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(self.graph):
             for l in range(w.n_layers):
-                p.flux_kv_append(l, w.batch, self.kn[l], self.vn[l], self.ktab[l], self.vtab[l], self.pos_cur)
-                p.flux_attn_decode(l, w.batch, self.q[l], self.ktab[l], self.vtab[l], self.ctx_cur, self.out[l])
+                p.flux_attn_decode_step(l, w.batch, self.q[l], self.kn[l], self.vn[l], self.ktab[l], self.vtab[l],
+                                        self.ctx_cur, self.out[l])
             self.ctx_cur += 1
             self.pos_cur += 1
         torch.cuda.synchronize()

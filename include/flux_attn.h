@@ -161,6 +161,18 @@ int flux_attn_decode(flux_plan *plan, int32_t layer, int32_t B, const void *q,
                      const void *const *k_caches, const void *const *v_caches,
                      const int32_t *ctx_len, void *out, void *stream);
 
+/* flux_kv_append and flux_attn_decode of one layer in one launch (Sec. 3.3: the new token's K, V
+ * join the cache, then the token attends): the kernel stores k_new / v_new at position
+ * ctx_len - 1 of each request's cache (ring slot for a compact sparse cache) and reads that one
+ * row from k_new / v_new instead of the cache, so no second kernel and no ordering between the
+ * two is needed.  Same results as the two calls with pos = ctx_len - 1.  At small batches the
+ * saved launch is a visible part of a decode step.
+ *   k_new, v_new  [B][n_kv_heads][head_dim], device.   Everything else as in flux_attn_decode;
+ *   requests with ctx_len <= 0 are skipped (nothing stored, zero output row). */
+int flux_attn_decode_step(flux_plan *plan, int32_t layer, int32_t B, const void *q,
+                          const void *k_new, const void *v_new, void *const *k_caches,
+                          void *const *v_caches, const int32_t *ctx_len, void *out, void *stream);
+
 /* Decode step for callers that cannot allocate device memory at all.  (The paper
  * has no counterpart: this is a packaging variant of flux_attn_decode, not part of
  * the method.)  Who needs it: code that runs inside a host program which owns all

@@ -514,6 +514,20 @@ int flux_attn_decode(flux_plan *plan, int32_t layer, int32_t B, const void *q,
     return launch_decode(plan, layer, B, q, k_caches, v_caches, ctx_len, out, (cudaStream_t)stream);
 }
 
+int flux_attn_decode_step(flux_plan *plan, int32_t layer, int32_t B, const void *q, const void *k_new,
+                          const void *v_new, void *const *k_caches, void *const *v_caches,
+                          const int32_t *ctx_len, void *out, void *stream)
+{
+    int rc = check_batch_call(plan, layer, B);
+    if (rc) return rc;
+    if (!q || !k_new || !v_new || !k_caches || !v_caches || !ctx_len || !out)
+        return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    if (!aligned16(q) || !aligned16(out) || !aligned16(k_new) || !aligned16(v_new))
+        return fail(FLUX_E_INVALID_ARG, "q / k_new / v_new / out must be 16-byte aligned");
+    return launch_decode(plan, layer, B, q, (const void *const *)k_caches, (const void *const *)v_caches, ctx_len,
+                         out, (cudaStream_t)stream, k_new, v_new);
+}
+
 int flux_attn_decode_host(flux_plan *plan, int32_t layer, int32_t B, const void *q_host,
                           const void *k_new_host, const void *v_new_host, void *const *k_caches,
                           void *const *v_caches, const int32_t *pos, const int32_t *ctx_len,

@@ -40,6 +40,9 @@ struct DecArgs {
     int32_t *sched;
     uint32_t *status;
     __nv_bfloat16 *out;
+    // fused append (flux_attn_decode_step): the newest token's K, V rows [B][Hkv][D]; NULL otherwise
+    const unsigned char *k_new;
+    const unsigned char *v_new;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -146,6 +149,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
     __shared__ int s_split[kMaxBatch];
     __shared__ int s_shift[kMaxBatch];
     __shared__ int s_units[kMaxBatch];
+    __shared__ int s_newrow[kMaxBatch];   // fused append: cache row of the newest token (-1: none)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int hpc = a.Hkv < kDecWarps ? a.Hkv : kDecWarps;
@@ -161,6 +165,12 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
         s_split[b] = r.split;
         s_shift[b] = r.shift;
         s_units[b] = (r.n_eff + cta_tok - 1) / cta_tok * n_hg;
+        {   // the newest token sits at position n - 1; in a compact sparse cache that is a ring slot
+            const bool compact = a.layout == FLUX_KV_COMPACT_SA && r.mode == 0;
+            const int pnew = r.n - 1;
+            s_newrow[b] = (a.k_new != nullptr && pnew >= 0)
+                              ? ((compact && pnew >= a.S) ? a.S + (pnew - a.S) % a.W : pnew) : -1;
+        }
         if (blockIdx.x == 0) {
             int32_t *d = a.debug + b * 8;
             d[0] = r.mode; d[1] = a.layer; d[2] = b; d[3] = r.n;
@@ -194,6 +204,23 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
     if (blockIdx.x == 0) {
         for (int b = tid; b <= a.B; b += blockDim.x) a.sched[b] = s_prefix[b];
         if (tid == 0) a.sched[a.B + 1] = span;
+    }
+    // fused append: CTA b stores request b's newest K, V rows into the caches.  Nothing in this
+    // launch reads those cache rows (the loaders below take them from k_new / v_new).
+    if (a.k_new != nullptr) {
+        const int row_u4 = a.Hkv * (kRowBytes / 16);
+        for (int b = blockIdx.x; b < a.B; b += gridDim.x) {
+            const int nr = s_newrow[b];
+            if (nr < 0) continue;
+            uint4 *kd = (uint4 *)const_cast<void *>(a.k_caches[b]) + (size_t)nr * row_u4;
+            uint4 *vd = (uint4 *)const_cast<void *>(a.v_caches[b]) + (size_t)nr * row_u4;
+            const uint4 *ks = (const uint4 *)a.k_new + (size_t)b * row_u4;
+            const uint4 *vs = (const uint4 *)a.v_new + (size_t)b * row_u4;
+            for (int i = tid; i < row_u4; i += blockDim.x) {
+                kd[i] = ks[i];
+                vd[i] = vs[i];
+            }
+        }
     }
     const int u_begin = blockIdx.x * span;
     const int u_end = min(total, u_begin + span);
@@ -247,6 +274,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
                 l_v = (const unsigned char *)a.v_caches[l_b];
             }
             const int n_eff = s_neff[l_b], split = s_split[l_b], shift = s_shift[l_b];
+            const int newrow = s_newrow[l_b];
             const int v0 = (lit.x * slices + slice) * kDecTile;
             const uint32_t sbase = my_smem_u32 + stage * kDecStageBytes;
 #pragma unroll
@@ -257,8 +285,14 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
                 const int pos = valid ? (v >= split ? v + shift : v) : 0;
                 const size_t off = ((size_t)pos * a.Hkv + head) * kRowBytes + lc * 16;
                 const uint32_t dst = sbase + r * kRowBytes + ((lc ^ (r & 7)) << 4);
-                cp_async16(dst, l_k + off, valid ? 16 : 0);
-                cp_async16(dst + kDecTile * kRowBytes, l_v + off, valid ? 16 : 0);
+                if (valid && pos == newrow) {   // the token being appended by this launch
+                    const size_t noff = ((size_t)l_b * a.Hkv + head) * kRowBytes + lc * 16;
+                    cp_async16(dst, a.k_new + noff, 16);
+                    cp_async16(dst + kDecTile * kRowBytes, a.v_new + noff, 16);
+                } else {
+                    cp_async16(dst, l_k + off, valid ? 16 : 0);
+                    cp_async16(dst + kDecTile * kRowBytes, l_v + off, valid ? 16 : 0);
+                }
             }
         }
         cp_async_commit();
@@ -511,7 +545,8 @@ int decode_setup(flux_plan *p)
 }
 
 int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *const *k_caches,
-                  const void *const *v_caches, const int32_t *ctx_len, void *out, cudaStream_t st)
+                  const void *const *v_caches, const int32_t *ctx_len, void *out, cudaStream_t st,
+                  const void *k_new, const void *v_new)
 {
     const flux_config &c = p->cfg;
     char *ws = (char *)p->ws;
@@ -530,6 +565,8 @@ int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *con
     a.sched = (int32_t *)(ws + p->lay.sched);
     a.status = (uint32_t *)(ws + p->lay.status);
     a.out = (__nv_bfloat16 *)out;
+    a.k_new = (const unsigned char *)k_new;
+    a.v_new = (const unsigned char *)v_new;
     const int rec = prof_begin(p, FLUX_KERNEL_DECODE, st);
     decode_kernel<<<p->dec_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
     prof_end(p, rec, st);
@@ -675,6 +712,8 @@ extern "C" int flux_attn_decode_noalloc(const flux_config *cfg, int32_t layer, i
     a.sched = (int32_t *)(ws + kNaOffSched);
     a.status = (uint32_t *)(ws + kNaOffStatus);
     a.out = (__nv_bfloat16 *)out;
+    a.k_new = nullptr;
+    a.v_new = nullptr;
     decode_kernel<<<nd->n_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
     rc = check_cuda(cudaGetLastError(), "decode kernel launch");
     if (rc) return rc;

@@ -308,6 +308,39 @@ def test_host_side_argument_errors_launch_nothing(flux):
     assert plan.flux_plan_status(raise_on_flag=False) == flux.FLUX_STATUS_BAD_LENGTH
 
 
+@pytest.mark.parametrize("layout", [0, 1])
+def test_fused_decode_step_equals_append_then_decode(flux, layout):
+    """flux_attn_decode_step must leave the same caches and give the same outputs, bit for bit, as
+    flux_kv_append followed by flux_attn_decode -- over several steps, so ring slots wrap."""
+    Hq, Hkv, S, W, L = 8, 2, 4, 8, 2
+    lens = [30, 9, 17, 0, 13]
+    B = len(lens)
+    plan = _plan(flux, L, Hq, Hkv, S, W, B, 64, layout)
+    mask = np.array([[1, 0], [0, 0], [1, 1], [0, 1], [0, 1]], dtype=np.uint8)
+    plan.flux_router_apply(mask=mask)
+    for layer in range(L):
+        rows = [S + W if (layout == 1 and mask[b, layer] == 0) else 64 for b in range(B)]
+        kc = [synth.normal_bf16((rows[b], Hkv, 128), 5, 10 * layer + b, DEV) for b in range(B)]
+        vc = [synth.normal_bf16((rows[b], Hkv, 128), 6, 10 * layer + b, DEV) for b in range(B)]
+        kc2 = [t.clone() for t in kc]; vc2 = [t.clone() for t in vc]
+        kt, vt = flux.pointer_table(kc, DEV), flux.pointer_table(vc, DEV)
+        kt2, vt2 = flux.pointer_table(kc2, DEV), flux.pointer_table(vc2, DEV)
+        for step in range(12):
+            n = [x + step if x > 0 else 0 for x in lens]
+            ctx = torch.tensor(n, dtype=torch.int32, device=DEV)
+            pos = torch.tensor([x - 1 for x in n], dtype=torch.int32, device=DEV)
+            q = synth.normal_bf16((B, Hq, 128), 7, 100 * layer + step, DEV)
+            kn = synth.normal_bf16((B, Hkv, 128), 8, 100 * layer + step, DEV)
+            vn = synth.normal_bf16((B, Hkv, 128), 9, 100 * layer + step, DEV)
+            plan.flux_kv_append(layer, B, kn, vn, kt, vt, pos)
+            want = plan.flux_attn_decode(layer, B, q, kt, vt, ctx)
+            got = plan.flux_attn_decode_step(layer, B, q, kn, vn, kt2, vt2, ctx)
+            assert torch.equal(got, want), (layer, step)
+        for b in range(B):
+            assert torch.equal(kc[b], kc2[b]) and torch.equal(vc[b], vc2[b]), (layer, b)
+    assert plan.flux_plan_status() == 0
+
+
 def test_decode_host_entry_point_matches_device_entry_point(flux):
     Hq, Hkv, S, W, B, L = 8, 2, 4, 8, 3, 2
     lens = [30, 9, 17]
