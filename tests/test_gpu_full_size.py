@@ -63,6 +63,31 @@ def test_prefill_full_size_sampled_rows(flux, cfg, kernel):
     assert plan.flux_plan_status() == 0
 
 
+def test_prefill_256k_in_chunks_sampled_rows(flux):
+    """The paper's headline length (Sec. 4.3: 256K tokens): Llama-3-8B attention shapes, sink 128 +
+    window 2048 (Table 3), prefilled in chunks of 16384 queries (Appendix D.3), one FA and one SA
+    layer; sampled rows of every chunk region against the oracle."""
+    N, Hq, Hkv, S, W, C = 262144, 32, 8, 128, 2048, 16384
+    plan = flux.Plan(flux.make_config(2, Hq, Hkv, S, W, 1, N), DEV)
+    plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
+    q = synth.normal_bf16((N, Hq, 128), 606, synth.stream_id("q"), DEV)
+    k = synth.normal_bf16((N, Hkv, 128), 606, synth.stream_id("k"), DEV)
+    v = synth.normal_bf16((N, Hkv, 128), 606, synth.stream_id("v"), DEV)
+    rows = np.unique(np.concatenate([synth.sample_rows(N, S, W, 12, 606),
+                                     np.array([C - 1, C, 5 * C + 77, N - C, N - C - 1])]))
+    heads = [0, 3, 4, 31]
+    rr = np.repeat(rows, len(heads))
+    hh = np.tile(np.asarray(heads, dtype=np.int64), len(rows))
+    qb, kb, vb = bits(q), bits(k), bits(v)
+    out = torch.empty_like(q)
+    for layer, mode in ((1, oracle.SA), (0, oracle.FA)):
+        for a in range(0, N, C):
+            plan.flux_attn_prefill(layer, 0, q[a:a + C], k[:a + C], v[:a + C], a, out[a:a + C])
+        ref = oracle.prefill_rows(mode, qb, kb, vb, 0, rr, hh, S, W, SCALE)
+        compare(out[torch.from_numpy(rr).to(DEV), torch.from_numpy(hh).to(DEV)], ref, "256K prefill mode %d" % mode)
+    assert plan.flux_plan_status() == 0
+
+
 @pytest.mark.parametrize("cfg", ["cfg3", "cfg4", "cfg5"])
 def test_decode_full_size_sampled(flux, cfg):
     """The decode workloads as bench.py builds them (compact sparse caches, per-request masks,
