@@ -1,8 +1,9 @@
 // Causal prefill of one routed layer on the sm_100a tensor cores (tcgen05 + TMEM + TMA).
 //
 // One CTA serves two query tiles at once: the same 128 query rows of two query
-// heads that share a KV head (GQA), so every K / V tile fetched by TMA feeds four
-// MMAs.  Roles (warp-specialised, three warpgroups):
+// heads that share a KV head (GQA) -- or, for a head left over by an odd group size (and
+// for plain multi-head attention), two consecutive row tiles of one head -- so every
+// K / V tile fetched by TMA feeds four MMAs.  Roles (warp-specialised, three warpgroups):
 //   warps 0-3   softmax of query tile 0 (one thread per query row, TMEM lane = row)
 //   warps 4-7   softmax of query tile 1
 //   warp  8     TMA producer: Q once, then K_j, V_j through a ring of shared-memory slots
@@ -67,7 +68,7 @@ struct TcArgs {
     __nv_bfloat16 *out;
     const uint8_t *mask;
     int L, layer, req, Hq, G, S, W, q_start, Nq;
-    int n_qt, ppg, n_pairs;
+    int n_qt, n_kv, P, odd;      // query tiles, KV heads, head pairs per KV head, 1 if a head is left over
     float scale_log2;
     int32_t *debug;
     uint32_t *status;
@@ -239,7 +240,11 @@ struct Cta {
     uint32_t tmem;          // TMEM base address
     volatile int *abort_flag;
     uint32_t *status;
-    int qt, kvh, h0, nslots, q_end, i0;
+    int kvh, nslots, q_end;
+    int head0, head1, qt0, qt1, i00, i01;   // per query tile: query head, tile index in the chunk, first absolute position
+    __device__ __forceinline__ int head(int t) const { return t ? head1 : head0; }
+    __device__ __forceinline__ int qt(int t) const { return t ? qt1 : qt0; }
+    __device__ __forceinline__ int i0(int t) const { return t ? i01 : i00; }
     int e1, b2, n_tiles;    // KV tiles kept: [0, e1) and [b2, b2 + n_tiles - e1)
     bool fa;
     __device__ __forceinline__ uint32_t bar(int i) const { return bar0 + 8u * (uint32_t)i; }
@@ -257,8 +262,8 @@ __device__ __forceinline__ void role_load(const Cta &c, const CUtensorMap *tm_q,
     if (elect_one()) {
         mbar_expect_tx(c.bar(BAR_Q_FULL), (uint32_t)(c.nslots * kTileBytes));
         for (int t = 0; t < c.nslots; ++t) {
-            tma_load_3d(c.sb + OFF_Q + t * kTileBytes, tm_q, c.bar(BAR_Q_FULL), 0, c.h0 + t, c.qt * BM);
-            tma_load_3d(c.sb + OFF_Q + t * kTileBytes + kHalfBytes, tm_q, c.bar(BAR_Q_FULL), 64, c.h0 + t, c.qt * BM);
+            tma_load_3d(c.sb + OFF_Q + t * kTileBytes, tm_q, c.bar(BAR_Q_FULL), 0, c.head(t), c.qt(t) * BM);
+            tma_load_3d(c.sb + OFF_Q + t * kTileBytes + kHalfBytes, tm_q, c.bar(BAR_Q_FULL), 64, c.head(t), c.qt(t) * BM);
         }
     }
     for (int it = 0; it < c.n_tiles; ++it) {
@@ -346,7 +351,8 @@ __device__ __forceinline__ void role_mma(const Cta &c)
 __device__ __forceinline__ void role_softmax(const Cta &c, const TcArgs &a, int t, int warp, int lane)
 {
     const int r = (warp & 3) * 32 + lane;            // row of the tile = TMEM lane
-    const int row = c.i0 + r;                        // absolute position of this query
+    const int i0 = c.i0(t);                          // first absolute position of this query tile
+    const int row = i0 + r;                          // absolute position of this query
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = c.tmem + lane_base + TM_S + t * 128;
     const uint32_t tO = c.tmem + lane_base + TM_O + t * 128;
@@ -363,7 +369,7 @@ __device__ __forceinline__ void role_softmax(const Cta &c, const TcArgs &a, int 
         tc_wait_ld();
         const int j0 = tile_of(it, c.e1, c.b2) * BN;
         const int jmax = j0 + BN - 1;
-        const bool full = (jmax <= c.i0) && (c.fa || jmax < S || j0 > c.i0 + BM - 1 - W);
+        const bool full = (jmax <= i0) && (c.fa || jmax < S || j0 > i0 + BM - 1 - W);
         if (!full) {
 #pragma unroll
             for (int q = 0; q < 4; ++q)
@@ -428,7 +434,7 @@ __device__ __forceinline__ void role_softmax(const Cta &c, const TcArgs &a, int 
     tc_fence_after();
     const float inv = 1.0f / (lsum.x + lsum.y);
     const bool valid = row < c.q_end;
-    __nv_bfloat16 *dst = a.out + ((size_t)(valid ? row - a.q_start : 0) * a.Hq + (c.h0 + t)) * kHeadDim;
+    __nv_bfloat16 *dst = a.out + ((size_t)(valid ? row - a.q_start : 0) * a.Hq + c.head(t)) * kHeadDim;
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
         uint32_t o[32];
@@ -471,15 +477,47 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
 
     // ---- which work item ----
     const int bid = blockIdx.x;
-    c.qt = a.n_qt - 1 - bid / a.n_pairs;                  // latest (heaviest) query tiles first
-    const int pr = bid % a.n_pairs;
-    c.kvh = pr / a.ppg;
-    const int pi = pr % a.ppg;
-    c.h0 = c.kvh * a.G + 2 * pi;
-    c.nslots = (2 * pi + 1 < a.G) ? 2 : 1;
+    // Work items, heaviest (latest query tiles) first.  An item is two query tiles that walk the
+    // same K / V tiles: the same 128 rows of two heads of a KV group, or -- for the head left
+    // over when the group size is odd -- two consecutive row tiles of that head (the earlier
+    // one simply finds its last KV tile fully masked).  Rank r = tiles counted from the end;
+    // ranks come in pairs (2k, 2k+1): n_kv * P head-pair items each, plus n_kv left-over items
+    // (tiles n_qt-1-2k and n_qt-2-2k) listed with the even rank.
+    {
+        const int per2 = a.n_kv * (2 * a.P + a.odd);
+        const int k2 = bid / per2;
+        int rem = bid % per2;
+        int r = 2 * k2;
+        bool leftover = false;
+        if (rem < a.n_kv * a.P) {
+        } else if (rem < a.n_kv * (a.P + a.odd)) {
+            leftover = true;
+            rem -= a.n_kv * a.P;
+        } else {
+            rem -= a.n_kv * (a.P + a.odd);
+            r += 1;
+        }
+        const int qt = a.n_qt - 1 - r;
+        if (!leftover) {
+            c.kvh = rem / a.P;
+            const int pi = rem % a.P;
+            c.head0 = c.kvh * a.G + 2 * pi;
+            c.head1 = c.head0 + 1;
+            c.qt0 = c.qt1 = qt;
+            c.nslots = 2;
+        } else {
+            c.kvh = rem;
+            c.head0 = c.head1 = c.kvh * a.G + a.G - 1;
+            c.qt0 = qt;
+            c.qt1 = qt - 1;
+            c.nslots = qt >= 1 ? 2 : 1;
+        }
+    }
     c.q_end = a.q_start + a.Nq;                           // KV rows present
-    c.i0 = a.q_start + c.qt * BM;
-    const int i_hi = min(c.i0 + BM - 1, c.q_end - 1);
+    c.i00 = a.q_start + c.qt0 * BM;
+    c.i01 = a.q_start + c.qt1 * BM;
+    const int i0_min = c.nslots == 2 ? c.i01 : c.i00;     // tile 1 is never later than tile 0
+    const int i_hi = min(c.i00 + BM - 1, c.q_end - 1);
 
     const uint8_t mode_raw = a.mask[a.req * a.L + a.layer];
     if (mode_raw > 1 && tid == 0) atomicOr(a.status, FLUX_STATUS_BAD_MASK);
@@ -499,7 +537,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         c.b2 = 0;
     } else {
         c.e1 = min((a.S + BN - 1) / BN, e2);
-        c.b2 = max(c.e1, max(0, c.i0 - a.W + 1) / BN);
+        c.b2 = max(c.e1, max(0, i0_min - a.W + 1) / BN);
     }
     c.n_tiles = c.e1 + max(0, e2 - c.b2);
 
@@ -640,13 +678,15 @@ int launch_prefill_tc(flux_plan *p, int layer, int req, const void *q, const voi
     a.L = c.n_layers; a.layer = layer; a.req = req; a.Hq = c.n_q_heads; a.G = p->G;
     a.S = c.sink; a.W = c.window; a.q_start = q_start; a.Nq = Nq;
     a.n_qt = (Nq + BM - 1) / BM;
-    a.ppg = (p->G + 1) / 2;
-    a.n_pairs = a.ppg * c.n_kv_heads;
+    a.n_kv = c.n_kv_heads;
+    a.P = p->G / 2;
+    a.odd = p->G & 1;
+    const int n_items = a.n_qt * a.n_kv * a.P + a.odd * a.n_kv * ((a.n_qt + 1) / 2);
     a.scale_log2 = p->scale_log2;
     a.debug = (int32_t *)(ws + p->lay.debug);
     a.status = (uint32_t *)(ws + p->lay.status);
     const int rec = prof_begin(p, FLUX_KERNEL_PREFILL, st);
-    prefill_tc_kernel<<<a.n_qt * a.n_pairs, kThreads, kSmemBytes, st>>>(tq, tk, tv, a);
+    prefill_tc_kernel<<<n_items, kThreads, kSmemBytes, st>>>(tq, tk, tv, a);
     prof_end(p, rec, st);
     p->launches++;
     p->debug_records = 1;

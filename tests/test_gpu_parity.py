@@ -125,6 +125,9 @@ PREFILL_CASES = [
     (520, 4, 1, 64, 256, (0, 512, 520)),
     (777, 6, 2, 130, 300, (0, 1, 129, 500, 777)),
     (1000, 3, 1, 0, 200, (0, 384, 1000)),
+    (300, 4, 4, 64, 100, None),           # one query head per KV head: a CTA pairs two row tiles of a head
+    (640, 5, 5, 128, 128, (0, 256, 640)),
+    (129, 1, 1, 5, 9, None),
 ]
 
 
