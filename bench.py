@@ -323,7 +323,7 @@ def prefill_block(flux, dev, peaks, warmup):
     ms_blk = e0.elapsed_time(e1) / 5
     off = bm.sum(axis=1).astype(np.int64) - 1                     # kept blocks below the diagonal, per query block
     pairs_blk = int((off * 64 * 64).sum() + nb * (64 * 65 // 2))  # + the causal half of each diagonal block
-    res["block_mask_sa"] = {"kernel": "prefill_blocks_kernel (mma.sync, 64 x 64 blocks)", "pattern":
+    res["block_mask_sa"] = {"kernel": "prefill_tc_kernel in block-mask mode (64 x 64 blocks inside 128 x 128 tiles)", "pattern":
                             "streaming at block granularity: %d sink + %d local blocks" % (-(-S // 64), -(-W // 64)),
                             "ms_layer": ms_blk, "tflops": 4 * Hq * D * pairs_blk / ms_blk / 1e9}
     if ms_fa is not None:

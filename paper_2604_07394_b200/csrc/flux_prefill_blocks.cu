@@ -271,7 +271,7 @@ int prefill_blocks_setup()
                       "cudaFuncSetAttribute(prefill_blocks_kernel)");
 }
 
-int launch_prefill_blocks(flux_plan *p, const void *q, const void *k, const void *v, int q_start, int Nq,
+int launch_prefill_blocks_mma(flux_plan *p, const void *q, const void *k, const void *v, int q_start, int Nq,
                           const uint8_t *block_mask, int n_kv_blocks, void *out, cudaStream_t st)
 {
     const flux_config &c = p->cfg;

@@ -72,6 +72,8 @@ struct TcArgs {
     float scale_log2;
     int32_t *debug;
     uint32_t *status;
+    const uint8_t *bm;           // block-mask mode: uint8 [absolute query block][n_kb], blocks of 64 positions
+    int n_kb;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -245,8 +247,10 @@ struct Cta {
     __device__ __forceinline__ int head(int t) const { return t ? head1 : head0; }
     __device__ __forceinline__ int qt(int t) const { return t ? qt1 : qt0; }
     __device__ __forceinline__ int i0(int t) const { return t ? i01 : i00; }
-    int e1, b2, n_tiles;    // KV tiles kept: [0, e1) and [b2, b2 + n_tiles - e1)
+    int e1, b2, n_tiles;    // routed layers: KV tiles kept are [0, e1) and [b2, b2 + n_tiles - e1)
     bool fa;
+    const uint8_t *bm;      // block-mask mode: mask, row length, last candidate KV tile
+    int n_kb, last_tile;
     __device__ __forceinline__ uint32_t bar(int i) const { return bar0 + 8u * (uint32_t)i; }
     // every lane of the (converged) calling warp waits; the result is the same for all of them
     __device__ __forceinline__ bool wait(int i, uint32_t parity) const
@@ -255,7 +259,63 @@ struct Cta {
     }
 };
 
+// The KV tiles of a work item, in the order every role walks them.  Called by all lanes of a
+// converged warp.  Routed FA / SA layers: a plain range.  Block-mask mode: the tiles [0, last_tile]
+// in which at least one kept 64 x 64 block meets the item's rows; the warp inspects 32 candidate
+// tiles at a time (one per lane) and hands out the non-empty ones.  pat: for query tile t, bit
+// 4 t + 2 rb + cb says that the block (row half rb, key half cb) of the 128 x 128 tile is kept.
+template <bool kBlock>
+struct TileWalk {
+    const Cta &c;
+    int it = 0, base = 0;
+    uint32_t bal = 0, mypat = 0;
+    __device__ __forceinline__ explicit TileWalk(const Cta &cta) : c(cta) {}
+    __device__ __forceinline__ uint32_t pattern(int j) const
+    {
+        uint32_t pat = 0;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            if (t >= c.nslots) break;
+#pragma unroll
+            for (int rb = 0; rb < 2; ++rb) {
+                const int qb = c.i0(t) / 64 + rb;
+                if (qb * 64 >= c.q_end) continue;
+#pragma unroll
+                for (int cb = 0; cb < 2; ++cb) {
+                    const int kb = 2 * j + cb;
+                    if (kb <= qb && kb < c.n_kb && c.bm[(size_t)qb * c.n_kb + kb] != 0) pat |= 1u << (4 * t + 2 * rb + cb);
+                }
+            }
+        }
+        return pat;
+    }
+    __device__ __forceinline__ bool next(int &jt, uint32_t &pat)
+    {
+        if (!kBlock) {
+            if (it >= c.n_tiles) return false;
+            jt = tile_of(it++, c.e1, c.b2);
+            pat = 0xffu;
+            return true;
+        }
+        const int lane = threadIdx.x & 31;
+        while (bal == 0) {
+            if (base > c.last_tile) return false;
+            const int j = base + lane;
+            mypat = j <= c.last_tile ? pattern(j) : 0u;
+            bal = __ballot_sync(0xffffffffu, mypat != 0u);
+            base += 32;
+        }
+        const int ln = __ffs(bal) - 1;
+        bal &= bal - 1;
+        jt = base - 32 + ln;
+        pat = __shfl_sync(0xffffffffu, mypat, ln);
+        ++it;
+        return true;
+    }
+};
+
 // ================= TMA producer (one warp, one issuing lane) =================
+template <bool kBlock>
 __device__ __forceinline__ void role_load(const Cta &c, const CUtensorMap *tm_q, const CUtensorMap *tm_k,
                                           const CUtensorMap *tm_v)
 {
@@ -266,8 +326,11 @@ __device__ __forceinline__ void role_load(const Cta &c, const CUtensorMap *tm_q,
             tma_load_3d(c.sb + OFF_Q + t * kTileBytes + kHalfBytes, tm_q, c.bar(BAR_Q_FULL), 64, c.head(t), c.qt(t) * BM);
         }
     }
-    for (int it = 0; it < c.n_tiles; ++it) {
-        const int j0 = tile_of(it, c.e1, c.b2) * BN;
+    TileWalk<kBlock> walk(c);
+    int jt;
+    uint32_t pat;
+    for (int it = 0; walk.next(jt, pat); ++it) {
+        const int j0 = jt * BN;
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
             const int qi = 2 * it + kv, slot = qi % kKvSlots, use = qi / kKvSlots;
@@ -287,6 +350,7 @@ __device__ __forceinline__ void role_load(const Cta &c, const CUtensorMap *tm_q,
 // Issue order per KV tile j:  PV_0[j] QK_0[j+1] PV_1[j] QK_1[j+1]; the tensor pipe runs them in
 // that order, so S_t[j+1] overwrites S_t / P_t only after PV_t[j] has read P_t[j].  (One issuer for
 // both tiles: two issuing warps, whose MMAs interleave instruction by instruction, ran slower.)
+template <bool kBlock>
 __device__ __forceinline__ void role_mma(const Cta &c)
 {
     // S_t = Q_t K^T, then up to two commits (tcgen05.commit belongs to the issuing lane; 0 = none)
@@ -317,15 +381,24 @@ __device__ __forceinline__ void role_mma(const Cta &c)
             if (bar_b) tc_commit(bar_b);
         }
     };
+    TileWalk<kBlock> walk(c);
+    int jt;
+    uint32_t pat;
+    bool more = walk.next(jt, pat);
     if (!c.wait(BAR_Q_FULL, 0)) return;
+    if (!more) {    // (block-mask mode) the item keeps no block at all: nothing to accumulate
+        if (elect_one())
+            for (int t = 0; t < c.nslots; ++t) tc_commit(c.bar(BAR_O_FULL + t));
+        return;
+    }
     if (!c.wait(BAR_KV_FULL + 0, 0)) return;
     tc_fence_after();
     for (int t = 0; t < c.nslots; ++t)
         qk(t, 0, c.bar(BAR_S_FULL + t), t == c.nslots - 1 ? c.bar(BAR_KV_EMPTY + 0) : 0u);
-    for (int it = 0; it < c.n_tiles; ++it) {
+    for (int it = 0; more; ++it) {
         const int vq = 2 * it + 1, vslot = vq % kKvSlots, vpar = (vq / kKvSlots) & 1;
         const int kq = 2 * it + 2, kslot = kq % kKvSlots, kpar = (kq / kKvSlots) & 1;
-        const bool more = it + 1 < c.n_tiles;
+        more = walk.next(jt, pat);
         if (!c.wait(BAR_KV_FULL + vslot, (uint32_t)vpar)) return;
         for (int t = 0; t < c.nslots; ++t) {
             const bool last = t == c.nslots - 1;
@@ -348,6 +421,7 @@ __device__ __forceinline__ void role_mma(const Cta &c)
 }
 
 // ================= softmax of query tile t (one thread per query row) =================
+template <bool kBlock>
 __device__ __forceinline__ void role_softmax(const Cta &c, const TcArgs &a, int t, int warp, int lane)
 {
     const int r = (warp & 3) * 32 + lane;            // row of the tile = TMEM lane
@@ -360,23 +434,30 @@ __device__ __forceinline__ void role_softmax(const Cta &c, const TcArgs &a, int 
     const float scale_log2 = a.scale_log2;
     float m_used = -INFINITY;                        // running maximum in use, scaled log2 units
     float2 lsum = make_float2(0.f, 0.f);
-    for (int it = 0; it < c.n_tiles; ++it) {
+    TileWalk<kBlock> walk(c);
+    int jt;
+    uint32_t pat;
+    for (int it = 0; walk.next(jt, pat); ++it) {
         if (!c.wait(BAR_S_FULL + t, (uint32_t)(it & 1))) return;
         tc_fence_after();
         uint32_t sr[4][32];
 #pragma unroll
         for (int q = 0; q < 4; ++q) tc_ld32(tS + q * 32, sr[q]);
         tc_wait_ld();
-        const int j0 = tile_of(it, c.e1, c.b2) * BN;
+        const int j0 = jt * BN;
         const int jmax = j0 + BN - 1;
-        const bool full = (jmax <= i0) && (c.fa || jmax < S || j0 > i0 + BM - 1 - W);
+        // this row's two block bits of the tile (block-mask mode): keys [j0, j0+64) and [j0+64, j0+128)
+        const uint32_t mine = pat >> (4 * t + 2 * (r >> 6));
+        const bool full = kBlock ? (jmax <= i0 && ((pat >> (4 * t)) & 0xfu) == 0xfu)
+                                 : ((jmax <= i0) && (c.fa || jmax < S || j0 > i0 + BM - 1 - W));
         if (!full) {
 #pragma unroll
             for (int q = 0; q < 4; ++q)
 #pragma unroll
                 for (int e = 0; e < 32; ++e) {
                     const int key = j0 + q * 32 + e;
-                    const bool keep = key <= row && (c.fa || key < S || key > row - W);
+                    const bool keep = kBlock ? (key <= row && ((mine >> (q >> 1)) & 1u) != 0u)
+                                             : (key <= row && (c.fa || key < S || key > row - W));
                     if (!keep) sr[q][e] = 0xff800000u;   // -inf
                 }
         }
@@ -432,7 +513,11 @@ __device__ __forceinline__ void role_softmax(const Cta &c, const TcArgs &a, int 
     }
     if (!c.wait(BAR_O_FULL + t, 0)) return;
     tc_fence_after();
-    const float inv = 1.0f / (lsum.x + lsum.y);
+    const float lrow = lsum.x + lsum.y;
+    // (block-mask mode) a row whose mask keeps no key: zero output row, flagged
+    const bool empty = kBlock && !(lrow > 0.f);
+    if (empty && row < c.q_end) atomicOr(c.status, FLUX_STATUS_BAD_MASK);
+    const float inv = empty ? 0.f : 1.0f / lrow;
     const bool valid = row < c.q_end;
     __nv_bfloat16 *dst = a.out + ((size_t)(valid ? row - a.q_start : 0) * a.Hq + c.head(t)) * kHeadDim;
 #pragma unroll
@@ -444,6 +529,10 @@ __device__ __forceinline__ void role_softmax(const Cta &c, const TcArgs &a, int 
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 uint4 w;
+                if (empty) {
+#pragma unroll
+                    for (int z = 0; z < 8; ++z) o[8 * e + z] = 0u;   // O holds nothing meaningful
+                }
                 w.x = pack_bf16(__uint_as_float(o[8 * e + 0]) * inv, __uint_as_float(o[8 * e + 1]) * inv);
                 w.y = pack_bf16(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv);
                 w.z = pack_bf16(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv);
@@ -454,6 +543,7 @@ __device__ __forceinline__ void role_softmax(const Cta &c, const TcArgs &a, int 
     }
 }
 
+template <bool kBlock>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                   const __grid_constant__ CUtensorMap tm_v, TcArgs a)
@@ -519,11 +609,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     const int i0_min = c.nslots == 2 ? c.i01 : c.i00;     // tile 1 is never later than tile 0
     const int i_hi = min(c.i00 + BM - 1, c.q_end - 1);
 
-    const uint8_t mode_raw = a.mask[a.req * a.L + a.layer];
+    const uint8_t mode_raw = kBlock ? (uint8_t)1 : a.mask[a.req * a.L + a.layer];
     if (mode_raw > 1 && tid == 0) atomicOr(a.status, FLUX_STATUS_BAD_MASK);
     c.fa = mode_raw != 0;
+    c.bm = a.bm;
+    c.n_kb = a.n_kb;
 
-    if (bid == 0 && tid == 0) {
+    if (!kBlock && bid == 0 && tid == 0) {
         const int n = c.q_end;
         const bool two = !c.fa && n > a.S + a.W;
         int32_t *d = a.debug;
@@ -540,6 +632,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         c.b2 = max(c.e1, max(0, i0_min - a.W + 1) / BN);
     }
     c.n_tiles = c.e1 + max(0, e2 - c.b2);
+    c.last_tile = e2 - 1;
 
     // ---- set-up: barriers, TMEM ----
     if (tid == 0) {
@@ -571,13 +664,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (warp >= 8) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
         if (warp == 8) {
-            role_load(c, &tm_q, &tm_k, &tm_v);
+            role_load<kBlock>(c, &tm_q, &tm_k, &tm_v);
         } else if (warp == 9) {
-            role_mma(c);
+            role_mma<kBlock>(c);
         }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
-        if (warp < 4 * c.nslots) role_softmax(c, a, warp >> 2, warp, lane);
+        if (warp < 4 * c.nslots) role_softmax<kBlock>(c, a, warp >> 2, warp, lane);
     }
 
     // ---- teardown ----
@@ -645,14 +738,19 @@ int prefill_tc_setup()
     }
     // setmaxnreg moves registers inside the CTA's own allocation (registers per thread at launch x
     // threads); a request beyond it would block for ever, so refuse to run rather than launch that.
-    cudaFuncAttributes fa;
-    int rc = check_cuda(cudaFuncGetAttributes(&fa, prefill_tc_kernel), "cudaFuncGetAttributes(prefill_tc_kernel)");
-    if (rc) return rc;
-    if (fa.numRegs * kThreads < 2 * kSoftmaxThreads * kSoftmaxRegs + (kThreads - 2 * kSoftmaxThreads) * kOtherRegs)
-        return fail(FLUX_E_CUDA, "prefill kernel was built with %d registers per thread: too few for its register rebalancing",
-                    fa.numRegs);
-    return check_cuda(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes),
-                      "cudaFuncSetAttribute(prefill_tc_kernel)");
+    for (int v = 0; v < 2; ++v) {
+        const void *fn = v ? (const void *)prefill_tc_kernel<true> : (const void *)prefill_tc_kernel<false>;
+        cudaFuncAttributes fa;
+        int rc = check_cuda(cudaFuncGetAttributes(&fa, fn), "cudaFuncGetAttributes(prefill_tc_kernel)");
+        if (rc) return rc;
+        if (fa.numRegs * kThreads < 2 * kSoftmaxThreads * kSoftmaxRegs + (kThreads - 2 * kSoftmaxThreads) * kOtherRegs)
+            return fail(FLUX_E_CUDA, "prefill kernel was built with %d registers per thread: too few for its register rebalancing",
+                        fa.numRegs);
+        rc = check_cuda(cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes),
+                        "cudaFuncSetAttribute(prefill_tc_kernel)");
+        if (rc) return rc;
+    }
+    return FLUX_OK;
 }
 
 int launch_wait_probe(flux_plan *p, long long limit_cycles, cudaStream_t st)
@@ -662,8 +760,9 @@ int launch_wait_probe(flux_plan *p, long long limit_cycles, cudaStream_t st)
     return check_cuda(cudaGetLastError(), "wait probe launch");
 }
 
+// block_mask == NULL: a routed layer (FA or SA by the cached routing bit); else block-mask mode
 int launch_prefill_tc(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v, int q_start,
-                      int Nq, void *out, cudaStream_t st)
+                      int Nq, void *out, cudaStream_t st, const uint8_t *block_mask, int n_kv_blocks)
 {
     const flux_config &c = p->cfg;
     char *ws = (char *)p->ws;
@@ -685,11 +784,16 @@ int launch_prefill_tc(flux_plan *p, int layer, int req, const void *q, const voi
     a.scale_log2 = p->scale_log2;
     a.debug = (int32_t *)(ws + p->lay.debug);
     a.status = (uint32_t *)(ws + p->lay.status);
+    a.bm = block_mask;
+    a.n_kb = n_kv_blocks;
     const int rec = prof_begin(p, FLUX_KERNEL_PREFILL, st);
-    prefill_tc_kernel<<<n_items, kThreads, kSmemBytes, st>>>(tq, tk, tv, a);
+    if (block_mask)
+        prefill_tc_kernel<true><<<n_items, kThreads, kSmemBytes, st>>>(tq, tk, tv, a);
+    else
+        prefill_tc_kernel<false><<<n_items, kThreads, kSmemBytes, st>>>(tq, tk, tv, a);
     prof_end(p, rec, st);
     p->launches++;
-    p->debug_records = 1;
+    if (!block_mask) p->debug_records = 1;
     return check_cuda(cudaGetLastError(), "prefill tensor-core kernel launch");
 }
 
