@@ -54,6 +54,22 @@ def traffic_note(kernel):
         return json.load(f).get(kernel)
 
 
+# ---- multi-rank bookkeeping (replicas: no data-path collective, only the timing reduction) -----
+
+def max_over_ranks(dist, values, device):
+    """Element-wise maximum of per-rank timings over all ranks (identity without a process group)."""
+    if dist is None:
+        return [float(v) for v in values]
+    tt = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+    return [float(v) for v in tt]
+
+
+def whole_job_throughput(world, units_per_rank_step, steps, ms_max):
+    """Units all ranks processed per second, over the slowest rank's time (weak scaling)."""
+    return world * units_per_rank_step * steps / (ms_max / 1e3)
+
+
 # ---- clocks ------------------------------------------------------------------------------------
 
 class ClockSampler:
@@ -620,14 +636,11 @@ def main():
         h1.record()
         barrier()
         e2e_ms = h0.elapsed_time(h1)
-    if dist is not None:
-        tt = torch.tensor([ms, e2e_ms if e2e_steps else 0.0], dtype=torch.float64, device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms, e2e_ms_max = float(tt[0]), float(tt[1])
-        if e2e_steps:
-            e2e_ms = e2e_ms_max
+    ms, e2e_ms_max = max_over_ranks(dist, [ms, e2e_ms if e2e_steps else 0.0], dev)
     if e2e_steps:
-        e2e = {"value": world * w.batch * e2e_steps / (e2e_ms / 1e3), "unit": "tokens/s",
+        e2e_ms = e2e_ms_max
+    if e2e_steps:
+        e2e = {"value": whole_job_throughput(world, w.batch, e2e_steps, e2e_ms), "unit": "tokens/s",
                "h2d_bytes_per_step": db.h2d_bytes(), "d2h_bytes_per_step": db.d2h_bytes(),
                "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
                "api": "flux_attn_decode_host per layer: pinned host q/k_new/v_new in, host out"}
@@ -638,7 +651,7 @@ def main():
             dist.destroy_process_group()
         return
 
-    value = world * w.batch * K_ / (ms / 1e3)
+    value = whole_job_throughput(world, w.batch, K_, ms)
     per_launch_bytes = roof_bytes / max(kcnt, 1)
     per_launch_ms = kms / max(kcnt, 1)
     ach = per_launch_bytes / (per_launch_ms * 1e-3) / 1e9
