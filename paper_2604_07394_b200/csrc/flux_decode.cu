@@ -470,10 +470,17 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
 }
 
 // Merge the partials of one (request, query head) and write the bf16 output row.
-__global__ void __launch_bounds__(128) decode_combine_kernel(DecArgs a)
+// Split-K combine: m = max m_p, l = sum l_p 2^(m_p - m), O = sum O_p 2^(m_p - m) / l over the
+// partials of one (request, query head).  One CTA per (request, head); its 16 warps take the
+// partials round-robin, four at a time with all loads issued before any is used (at batch 1 one
+// head has a few hundred partials, and a loop of dependent loads would cost more than the decode
+// kernel itself), then the warps' results are merged through shared memory.
+constexpr int kCombWarps = 16;
+
+__global__ void __launch_bounds__(kCombWarps * 32) decode_combine_kernel(DecArgs a)
 {
-    __shared__ float s_o[4][kHeadDim];
-    __shared__ float s_m[4], s_l[4];
+    __shared__ float s_o[kCombWarps][kHeadDim];
+    __shared__ float s_m[kCombWarps], s_l[kCombWarps];
     const int b = blockIdx.x / a.Hq, h = blockIdx.x % a.Hq;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int hpc = a.Hkv < kDecWarps ? a.Hkv : kDecWarps;
@@ -484,7 +491,7 @@ __global__ void __launch_bounds__(128) decode_combine_kernel(DecArgs a)
     const int ustart = a.sched[b], uend = a.sched[b + 1], span = a.sched[a.B + 1];
     const int units = uend - ustart;
     if (units == 0) {  // inactive request
-        dst[threadIdx.x] = __float2bfloat16(0.f);
+        if (threadIdx.x < kHeadDim) dst[threadIdx.x] = __float2bfloat16(0.f);
         return;
     }
     const int tiles = units / n_hg;
@@ -497,19 +504,41 @@ __global__ void __launch_bounds__(128) decode_combine_kernel(DecArgs a)
 
     float m = kNegBig, l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int p = warp; p < n_part; p += 4) {
-        const int c = c_first + p / slices, s = p % slices;
-        const size_t slot = ((size_t)c + seg) * kDecWarps + (hw + hpc * s);
-        const float *pm = a.part_ml + (slot * a.G + r) * 2;
-        const float mp = pm[0], lp = pm[1];
-        const float4 op = *reinterpret_cast<const float4 *>(a.part_o + (slot * a.G + r) * kHeadDim + lane * 4);
-        const float m_new = fmaxf(m, mp);
-        const float so = fast_exp2(m - m_new), sp = fast_exp2(mp - m_new);
-        acc.x = acc.x * so + op.x * sp;
-        acc.y = acc.y * so + op.y * sp;
-        acc.z = acc.z * so + op.z * sp;
-        acc.w = acc.w * so + op.w * sp;
-        l = l * so + lp * sp;
+    constexpr int kUnroll = 4;
+    for (int p0 = warp; p0 < n_part; p0 += kCombWarps * kUnroll) {
+        float mp[kUnroll], lp[kUnroll];
+        float4 op[kUnroll];
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const int p = p0 + u * kCombWarps;
+            if (p < n_part) {
+                const int c = c_first + p / slices, sl = p % slices;
+                const size_t slot = ((size_t)c + seg) * kDecWarps + (hw + hpc * sl);
+                const float2 ml = *reinterpret_cast<const float2 *>(a.part_ml + (slot * a.G + r) * 2);
+                mp[u] = ml.x;
+                lp[u] = ml.y;
+                op[u] = *reinterpret_cast<const float4 *>(a.part_o + (slot * a.G + r) * kHeadDim + lane * 4);
+            } else {
+                mp[u] = kNegBig;
+                lp[u] = 0.f;
+                op[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        float m_new = m;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) m_new = fmaxf(m_new, mp[u]);
+        const float so = fast_exp2(m - m_new);
+        acc.x *= so; acc.y *= so; acc.z *= so; acc.w *= so;
+        l *= so;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) {
+            const float sp = fast_exp2(mp[u] - m_new);
+            acc.x += op[u].x * sp;
+            acc.y += op[u].y * sp;
+            acc.z += op[u].z * sp;
+            acc.w += op[u].w * sp;
+            l += lp[u] * sp;
+        }
         m = m_new;
     }
     *reinterpret_cast<float4 *>(&s_o[warp][lane * 4]) = acc;
@@ -518,11 +547,14 @@ __global__ void __launch_bounds__(128) decode_combine_kernel(DecArgs a)
         s_l[warp] = l;
     }
     __syncthreads();
+    if (threadIdx.x >= kHeadDim) return;
     const int d = threadIdx.x;
-    float mm = fmaxf(fmaxf(s_m[0], s_m[1]), fmaxf(s_m[2], s_m[3]));
+    float mm = kNegBig;
+#pragma unroll
+    for (int w = 0; w < kCombWarps; ++w) mm = fmaxf(mm, s_m[w]);
     float num = 0.f, den = 0.f;
 #pragma unroll
-    for (int w = 0; w < 4; ++w) {
+    for (int w = 0; w < kCombWarps; ++w) {
         const float sc = fast_exp2(s_m[w] - mm);
         num += s_o[w][d] * sc;
         den += s_l[w] * sc;
@@ -573,7 +605,7 @@ int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *con
     p->launches++;
     int rc = check_cuda(cudaGetLastError(), "decode kernel launch");
     if (rc) return rc;
-    decode_combine_kernel<<<B * c.n_q_heads, 128, 0, st>>>(a);
+    decode_combine_kernel<<<B * c.n_q_heads, kCombWarps * 32, 0, st>>>(a);
     p->launches++;
     p->debug_records = B;
     return check_cuda(cudaGetLastError(), "decode combine kernel launch");
@@ -717,7 +749,7 @@ extern "C" int flux_attn_decode_noalloc(const flux_config *cfg, int32_t layer, i
     decode_kernel<<<nd->n_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
     rc = check_cuda(cudaGetLastError(), "decode kernel launch");
     if (rc) return rc;
-    decode_combine_kernel<<<B * cfg->n_q_heads, 128, 0, st>>>(a);
+    decode_combine_kernel<<<B * cfg->n_q_heads, kCombWarps * 32, 0, st>>>(a);
     rc = check_cuda(cudaGetLastError(), "decode combine kernel launch");
     if (rc) return rc;
     if (status_out)
