@@ -231,6 +231,15 @@ int flux_plan_status(flux_plan *plan, uint32_t *status_bits, void *stream);
 int flux_debug_dispatch(flux_plan *plan, int32_t *records_out, int32_t max_records,
                         int32_t *n_records_out, void *stream);
 
+/* Which KV rows the kernels actually read, for verification.  While a bitmap is set, the decode
+ * kernel sets bit r of request b's words for every cache row r (slot, in a compact sparse cache)
+ * whose K and V it loads, and the tcgen05 prefill kernel sets the bits of every position of every
+ * KV tile it loads (request words 0; tiles are 128 positions, clipped to the rows present).
+ *   bitmap  uint32 [max_batch][words_per_request], device, zeroed by the caller; NULL turns the
+ *           recording off (the default).  words_per_request * 32 >= max_context.
+ * The bits accumulate over launches until the caller clears the buffer. */
+int flux_debug_touched(flux_plan *plan, uint32_t *bitmap, int32_t words_per_request);
+
 /* Per-kernel device timing for roofline reports.  flux_profile_enable creates
  * max_records pairs of CUDA events (host objects; max_records == 0 turns
  * profiling off and destroys them); while enabled, every launch of a dominant

@@ -302,6 +302,8 @@ int flux_plan_create(const flux_config *cfg, flux_plan **plan)
     p->mask_B = 0;
     p->launches = 0;
     p->debug_records = 0;
+    p->touch = nullptr;
+    p->touch_words = 0;
     p->prof_ev = nullptr;
     p->prof_kind = nullptr;
     p->prof_cap = p->prof_n = 0;
@@ -437,6 +439,17 @@ int flux_attn_prefill_blocks(flux_plan *plan, const void *q, const void *k, cons
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(out))
         return fail(FLUX_E_INVALID_ARG, "tensor pointers must be 16-byte aligned");
     return launch_prefill_blocks(plan, q, k, v, q_start, Nq, block_mask, n_kv_blocks, out, (cudaStream_t)stream);
+}
+
+int flux_debug_touched(flux_plan *plan, uint32_t *bitmap, int32_t words_per_request)
+{
+    int rc = need_plan(plan, false);
+    if (rc) return rc;
+    if (bitmap && (words_per_request < 1 || (int64_t)words_per_request * 32 < plan->cfg.max_context))
+        return fail(FLUX_E_INVALID_ARG, "the bitmap needs one bit per position up to max_context");
+    plan->touch = bitmap;
+    plan->touch_words = bitmap ? words_per_request : 0;
+    return FLUX_OK;
 }
 
 int flux_debug_wait_probe(flux_plan *plan, int64_t limit_cycles, void *stream)

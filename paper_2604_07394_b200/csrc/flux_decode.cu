@@ -43,6 +43,8 @@ struct DecArgs {
     // fused append (flux_attn_decode_step): the newest token's K, V rows [B][Hkv][D]; NULL otherwise
     const unsigned char *k_new;
     const unsigned char *v_new;
+    uint32_t *touch;            // debug bitmap of the cache rows read ([B][touch_words]), or NULL
+    int touch_words;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -285,6 +287,8 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
                 const int pos = valid ? (v >= split ? v + shift : v) : 0;
                 const size_t off = ((size_t)pos * a.Hkv + head) * kRowBytes + lc * 16;
                 const uint32_t dst = sbase + r * kRowBytes + ((lc ^ (r & 7)) << 4);
+                if (a.touch != nullptr && valid && lc == 0 && head == 0)
+                    atomicOr(a.touch + (size_t)l_b * a.touch_words + (pos >> 5), 1u << (pos & 31));
                 if (valid && pos == newrow) {   // the token being appended by this launch
                     const size_t noff = ((size_t)l_b * a.Hkv + head) * kRowBytes + lc * 16;
                     cp_async16(dst, a.k_new + noff, 16);
@@ -599,6 +603,8 @@ int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *con
     a.out = (__nv_bfloat16 *)out;
     a.k_new = (const unsigned char *)k_new;
     a.v_new = (const unsigned char *)v_new;
+    a.touch = p->touch;
+    a.touch_words = p->touch_words;
     const int rec = prof_begin(p, FLUX_KERNEL_DECODE, st);
     decode_kernel<<<p->dec_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
     prof_end(p, rec, st);
@@ -746,6 +752,8 @@ extern "C" int flux_attn_decode_noalloc(const flux_config *cfg, int32_t layer, i
     a.out = (__nv_bfloat16 *)out;
     a.k_new = nullptr;
     a.v_new = nullptr;
+    a.touch = nullptr;
+    a.touch_words = 0;
     decode_kernel<<<nd->n_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
     rc = check_cuda(cudaGetLastError(), "decode kernel launch");
     if (rc) return rc;

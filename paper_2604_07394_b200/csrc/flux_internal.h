@@ -70,6 +70,8 @@ struct flux_plan {
     int32_t mask_B;
     int64_t launches;
     int32_t debug_records;  // records the latest call wrote
+    uint32_t *touch;        // optional device bitmap of the KV rows read (flux_debug_touched), NULL = off
+    int32_t touch_words;    // 32-bit words per request
     int dec_ctas;
     int prefill_kernel;     // FLUX_PREFILL_*
     // optional per-kernel timing (host-side event pool)

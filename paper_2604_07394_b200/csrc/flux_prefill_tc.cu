@@ -74,6 +74,7 @@ struct TcArgs {
     uint32_t *status;
     const uint8_t *bm;           // block-mask mode: uint8 [absolute query block][n_kb], blocks of 64 positions
     int n_kb;
+    uint32_t *touch;             // debug bitmap of the KV positions loaded, or NULL
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -317,7 +318,7 @@ struct TileWalk {
 // ================= TMA producer (one warp, one issuing lane) =================
 template <bool kBlock>
 __device__ __forceinline__ void role_load(const Cta &c, const CUtensorMap *tm_q, const CUtensorMap *tm_k,
-                                          const CUtensorMap *tm_v)
+                                          const CUtensorMap *tm_v, uint32_t *touch)
 {
     if (elect_one()) {
         mbar_expect_tx(c.bar(BAR_Q_FULL), (uint32_t)(c.nslots * kTileBytes));
@@ -331,6 +332,11 @@ __device__ __forceinline__ void role_load(const Cta &c, const CUtensorMap *tm_q,
     uint32_t pat;
     for (int it = 0; walk.next(jt, pat); ++it) {
         const int j0 = jt * BN;
+        if (touch != nullptr) {   // debug: the positions of this tile that exist, 32 per lane 0..3
+            const int lane = threadIdx.x & 31, first = j0 + 32 * lane;
+            if (lane < 4 && first < c.q_end)
+                atomicOr(touch + (first >> 5), c.q_end - first >= 32 ? 0xffffffffu : (1u << (c.q_end - first)) - 1u);
+        }
 #pragma unroll
         for (int kv = 0; kv < 2; ++kv) {
             const int qi = 2 * it + kv, slot = qi % kKvSlots, use = qi / kKvSlots;
@@ -664,7 +670,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (warp >= 8) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
         if (warp == 8) {
-            role_load<kBlock>(c, &tm_q, &tm_k, &tm_v);
+            role_load<kBlock>(c, &tm_q, &tm_k, &tm_v, a.touch);
         } else if (warp == 9) {
             role_mma<kBlock>(c);
         }
@@ -786,6 +792,7 @@ int launch_prefill_tc(flux_plan *p, int layer, int req, const void *q, const voi
     a.status = (uint32_t *)(ws + p->lay.status);
     a.bm = block_mask;
     a.n_kb = n_kv_blocks;
+    a.touch = p->touch;
     const int rec = prof_begin(p, FLUX_KERNEL_PREFILL, st);
     if (block_mask)
         prefill_tc_kernel<true><<<n_items, kThreads, kSmemBytes, st>>>(tq, tk, tv, a);

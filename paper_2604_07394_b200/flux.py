@@ -45,7 +45,7 @@ EXPORTS = [
     "flux_plan_create", "flux_plan_destroy", "flux_workspace_size", "flux_plan_set_workspace",
     "flux_router_apply", "flux_attn_prefill", "flux_attn_prefill_blocks", "flux_kv_retain", "flux_kv_append",
     "flux_attn_decode", "flux_attn_decode_step", "flux_attn_decode_noalloc", "flux_attn_decode_host", "flux_attn_prefill_host", "flux_plan_status",
-    "flux_debug_dispatch", "flux_debug_prefill_kernel", "flux_debug_wait_probe", "flux_profile_enable", "flux_profile_read", "flux_launch_count", "flux_last_error", "flux_version",
+    "flux_debug_dispatch", "flux_debug_touched", "flux_debug_prefill_kernel", "flux_debug_wait_probe", "flux_profile_enable", "flux_profile_read", "flux_launch_count", "flux_last_error", "flux_version",
 ]
 
 
@@ -96,6 +96,7 @@ def load():
     L.flux_plan_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
     L.flux_debug_dispatch.argtypes = [vp, vp, i32, ctypes.POINTER(i32), vp]
     L.flux_debug_prefill_kernel.argtypes = [vp, i32]
+    L.flux_debug_touched.argtypes = [vp, vp, i32]
     L.flux_debug_wait_probe.argtypes = [vp, ctypes.c_int64, vp]
     L.flux_profile_enable.argtypes = [vp, i32]
     L.flux_profile_read.argtypes = [vp, i32, ctypes.POINTER(ctypes.c_double),
@@ -254,6 +255,12 @@ class Plan:
         n = ctypes.c_int32()
         _check(load().flux_debug_dispatch(self._h, rec.ctypes.data, max_records, ctypes.byref(n), _stream()))
         return rec[: n.value].copy()
+
+    def flux_debug_touched(self, bitmap=None) -> None:
+        """bitmap: int32/uint32 device tensor [max_batch][words] (zeroed by the caller) or None (off)."""
+        words = 0 if bitmap is None else int(bitmap.shape[1])
+        _check(load().flux_debug_touched(self._h, _ptr(bitmap), words))
+        self._touch = bitmap          # keep it alive while the plan points at it
 
     def flux_debug_wait_probe(self, limit_cycles: int) -> None:
         _check(load().flux_debug_wait_probe(self._h, limit_cycles, _stream()))

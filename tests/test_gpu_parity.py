@@ -239,6 +239,77 @@ def test_decode_small_shapes(flux, Hq, Hkv, S, W, lens, layout):
     assert plan.flux_plan_status() == 0
 
 
+# ---- the KV rows the kernels read, bit for bit --------------------------------------------------
+
+def _bits_set(words):
+    w = words.cpu().numpy().astype(np.uint32)
+    return np.nonzero(np.unpackbits(w.view(np.uint8), bitorder="little"))[0].tolist()
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_decode_reads_exactly_the_kept_rows(flux, layout):
+    """Every cache row whose K / V the decode kernel loads is recorded in a bitmap; per request the
+    set must equal the oracle's kept set (mapped through the ring-slot rule for compact caches)."""
+    Hq, Hkv, S, W, L = 8, 2, 16, 48, 2
+    lens = [300, 64, 65, 5, 0, 1000]
+    B = len(lens)
+    cap = 1024
+    mask = np.array([[1, 0], [0, 1], [0, 0], [0, 1], [1, 0], [0, 0]], dtype=np.uint8)
+    plan = _plan(flux, L, Hq, Hkv, S, W, B, cap, layout)
+    plan.flux_router_apply(mask=mask)
+    touched = torch.zeros((B, cap // 32), dtype=torch.int32, device=DEV)
+    plan.flux_debug_touched(touched)
+    for layer in range(L):
+        rows = [S + W if (layout == 1 and mask[b, layer] == 0) else cap for b in range(B)]
+        kc = [synth.normal_bf16((rows[b], Hkv, 128), 3, 10 * layer + b, DEV) for b in range(B)]
+        vc = [synth.normal_bf16((rows[b], Hkv, 128), 4, 10 * layer + b, DEV) for b in range(B)]
+        q = synth.normal_bf16((B, Hq, 128), 5, layer, DEV)
+        ctx = torch.tensor(lens, dtype=torch.int32, device=DEV)
+        touched.zero_()
+        plan.flux_attn_decode(layer, B, q, flux.pointer_table(kc, DEV), flux.pointer_table(vc, DEV), ctx)
+        torch.cuda.synchronize()
+        for b, n in enumerate(lens):
+            got = _bits_set(touched[b])
+            if n == 0:
+                assert got == []
+                continue
+            mode = int(mask[b, layer])
+            want = oracle.kept(mode, n - 1, S, W).tolist()
+            if layout == 1 and mode == 0:
+                want = sorted(oracle.compact_slot(int(j), S, W) for j in want)
+            assert got == want, (layer, b, n, mode)
+    plan.flux_debug_touched(None)
+    assert plan.flux_plan_status() == 0
+
+
+def test_prefill_chunk_loads_exactly_the_tiles_its_rows_keep(flux):
+    """A late chunk of a prompt: the 128-position KV tiles the tcgen05 kernel loads are exactly the
+    tiles that hold a position some row of the chunk keeps (sink tiles + window tiles for SA,
+    everything up to the chunk's end for FA)."""
+    N, Hq, Hkv, S, W, q0 = 1000, 4, 2, 64, 200, 512
+    plan = _plan(flux, 2, Hq, Hkv, S, W, 1, 1024)
+    plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
+    q = synth.normal_bf16((N - q0, Hq, 128), 9, 1, DEV)
+    k = synth.normal_bf16((N, Hkv, 128), 9, 2, DEV)
+    v = synth.normal_bf16((N, Hkv, 128), 9, 3, DEV)
+    touched = torch.zeros((1, 1024 // 32), dtype=torch.int32, device=DEV)
+    plan.flux_debug_touched(touched)
+    for layer, mode in ((0, oracle.FA), (1, oracle.SA)):
+        touched.zero_()
+        out = plan.flux_attn_prefill(layer, 0, q, k, v, q0)
+        torch.cuda.synchronize()
+        kept = set()
+        for i in range(q0, N):
+            kept.update(oracle.kept(mode, i, S, W).tolist())
+        tiles = sorted({j // 128 for j in kept})
+        want = [j for t in tiles for j in range(128 * t, min(N, 128 * t + 128))]
+        assert _bits_set(touched[0]) == want, mode
+        ref = oracle.prefill(mode, bits(q), bits(k), bits(v), q0, S, W, _scale())
+        compare(out, ref, "late chunk mode %d" % mode)
+    plan.flux_debug_touched(None)
+    assert plan.flux_plan_status() == 0
+
+
 # ---- routing and error behaviour ---------------------------------------------------------------
 
 def test_router_inputs_and_device_flags(flux):
