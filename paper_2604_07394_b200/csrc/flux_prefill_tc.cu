@@ -44,10 +44,11 @@ constexpr int kSoftmaxRegs = 224, kOtherRegs = 56;   // per-thread register targ
 constexpr int OFF_Q = 0;                          // Q tile 0, Q tile 1
 constexpr int OFF_KV = 2 * kTileBytes;
 constexpr int OFF_BAR = OFF_KV + kKvSlots * kTileBytes;
-// mbarriers: Q_FULL | KV_FULL[slots] | KV_EMPTY[slots] | S_FULL[2] | P_FULL[tile][half] | O_FULL[2]
+// mbarriers: Q_FULL | KV_FULL[slots] | KV_EMPTY[slots] | S_FULL[2] | P_FULL[tile][half] | O_FULL[2] |
+//            Q_EMPTY   (hands the Q tiles over from one work item to the next)
 constexpr int BAR_Q_FULL = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = BAR_KV_FULL + kKvSlots,
               BAR_S_FULL = BAR_KV_EMPTY + kKvSlots, BAR_P_FULL = BAR_S_FULL + 2, BAR_O_FULL = BAR_P_FULL + 4,
-              kNumBars = BAR_O_FULL + 2;
+              BAR_Q_EMPTY = BAR_O_FULL + 2, kNumBars = BAR_Q_EMPTY + 1;
 static_assert(kNumBars <= 24, "barrier area");
 constexpr int OFF_TMEM_PTR = OFF_BAR + 24 * 8;
 constexpr int OFF_ABORT = OFF_TMEM_PTR + 4;
@@ -69,6 +70,7 @@ struct TcArgs {
     const uint8_t *mask;
     int L, layer, req, Hq, G, S, W, q_start, Nq;
     int n_qt, n_kv, P, odd;      // query tiles, KV heads, head pairs per KV head, 1 if a head is left over
+    int n_items;                 // work items of the launch
     float scale_log2;
     int32_t *debug;
     uint32_t *status;
@@ -226,6 +228,12 @@ __device__ __forceinline__ float2 fadd2(float2 a, float2 b)
         : "l"(reinterpret_cast<uint64_t const &>(a)), "l"(reinterpret_cast<uint64_t const &>(b)));
     return d;
 }
+// One 32-byte store (a whole sector per thread; the address is 32-byte aligned)
+__device__ __forceinline__ void st_global_32B(void *ptr, const uint32_t (&w)[8])
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(ptr), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                 "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     uint32_t r;
@@ -259,6 +267,67 @@ struct Cta {
         return __all_sync(0xffffffffu, mbar_wait(bar(i), parity, abort_flag, status));
     }
 };
+
+// Work items, heaviest (latest query tiles) first.  An item is two query tiles that walk the
+// same K / V tiles: the same 128 rows of two heads of a KV group, or -- for the head left
+// over when the group size is odd -- two consecutive row tiles of that head (the earlier
+// one simply finds its last KV tile fully masked).  Rank r = tiles counted from the end;
+// ranks come in pairs (2k, 2k+1): n_kv * P head-pair items each, plus n_kv left-over items
+// (tiles n_qt-1-2k and n_qt-2-2k) listed with the even rank.
+__device__ __forceinline__ void decode_item(const TcArgs &a, int item, bool fa, Cta &c)
+{
+    const int per2 = a.n_kv * (2 * a.P + a.odd);
+    const int k2 = item / per2;
+    int rem = item % per2;
+    int r = 2 * k2;
+    bool leftover = false;
+    if (rem < a.n_kv * a.P) {
+    } else if (rem < a.n_kv * (a.P + a.odd)) {
+        leftover = true;
+        rem -= a.n_kv * a.P;
+    } else {
+        rem -= a.n_kv * (a.P + a.odd);
+        r += 1;
+    }
+    const int qt = a.n_qt - 1 - r;
+    if (!leftover) {
+        c.kvh = rem / a.P;
+        const int pi = rem % a.P;
+        c.head0 = c.kvh * a.G + 2 * pi;
+        c.head1 = c.head0 + 1;
+        c.qt0 = c.qt1 = qt;
+        c.nslots = 2;
+    } else {
+        c.kvh = rem;
+        c.head0 = c.head1 = c.kvh * a.G + a.G - 1;
+        c.qt0 = qt;
+        c.qt1 = qt - 1;
+        c.nslots = qt >= 1 ? 2 : 1;
+    }
+    c.i00 = a.q_start + c.qt0 * BM;
+    c.i01 = a.q_start + c.qt1 * BM;
+    const int i0_min = c.nslots == 2 ? c.i01 : c.i00;     // tile 1 is never later than tile 0
+    const int i_hi = min(c.i00 + BM - 1, c.q_end - 1);
+    const int e2 = i_hi / BN + 1;
+    if (fa) {
+        c.e1 = 0;
+        c.b2 = 0;
+    } else {
+        c.e1 = min((a.S + BN - 1) / BN, e2);
+        c.b2 = max(c.e1, max(0, i0_min - a.W + 1) / BN);
+    }
+    c.n_tiles = c.e1 + max(0, e2 - c.b2);
+    c.last_tile = e2 - 1;
+}
+
+// The kernel is persistent: CTA b of G takes items b, 2G-1-b, 2G+b, 4G-1-b, ... (a serpentine over
+// the weight-sorted list, so every CTA gets nearly the same amount of work).  Returns the k-th item
+// of this CTA, or a number >= n_items when there is none.
+__device__ __forceinline__ int item_of(int k)
+{
+    const int G = (int)gridDim.x, b = (int)blockIdx.x;
+    return k * G + ((k & 1) ? G - 1 - b : b);
+}
 
 // The KV tiles of a work item, in the order every role walks them.  Called by all lanes of a
 // converged warp.  Routed FA / SA layers: a plain range.  Block-mask mode: the tiles [0, last_tile]
@@ -317,36 +386,44 @@ struct TileWalk {
 
 // ================= TMA producer (one warp, one issuing lane) =================
 template <bool kBlock>
-__device__ __forceinline__ void role_load(const Cta &c, const CUtensorMap *tm_q, const CUtensorMap *tm_k,
-                                          const CUtensorMap *tm_v, uint32_t *touch)
+__device__ __forceinline__ void role_load(Cta &c, const TcArgs &a, const CUtensorMap *tm_q, const CUtensorMap *tm_k,
+                                          const CUtensorMap *tm_v)
 {
-    if (elect_one()) {
-        mbar_expect_tx(c.bar(BAR_Q_FULL), (uint32_t)(c.nslots * kTileBytes));
-        for (int t = 0; t < c.nslots; ++t) {
-            tma_load_3d(c.sb + OFF_Q + t * kTileBytes, tm_q, c.bar(BAR_Q_FULL), 0, c.head(t), c.qt(t) * BM);
-            tma_load_3d(c.sb + OFF_Q + t * kTileBytes + kHalfBytes, tm_q, c.bar(BAR_Q_FULL), 64, c.head(t), c.qt(t) * BM);
+    int qi = 0;                                      // K / V tiles requested so far (ring position)
+    for (int k = 0;; ++k) {
+        const int item = item_of(k);
+        if (item >= a.n_items) break;
+        decode_item(a, item, c.fa, c);
+        // Q of the next item may overwrite Q of this one once its last QK^T has completed
+        if (k > 0 && !c.wait(BAR_Q_EMPTY, (uint32_t)((k - 1) & 1))) return;
+        if (elect_one()) {
+            mbar_expect_tx(c.bar(BAR_Q_FULL), (uint32_t)(c.nslots * kTileBytes));
+            for (int t = 0; t < c.nslots; ++t) {
+                tma_load_3d(c.sb + OFF_Q + t * kTileBytes, tm_q, c.bar(BAR_Q_FULL), 0, c.head(t), c.qt(t) * BM);
+                tma_load_3d(c.sb + OFF_Q + t * kTileBytes + kHalfBytes, tm_q, c.bar(BAR_Q_FULL), 64, c.head(t), c.qt(t) * BM);
+            }
         }
-    }
-    TileWalk<kBlock> walk(c);
-    int jt;
-    uint32_t pat;
-    for (int it = 0; walk.next(jt, pat); ++it) {
-        const int j0 = jt * BN;
-        if (touch != nullptr) {   // debug: the positions of this tile that exist, 32 per lane 0..3
-            const int lane = threadIdx.x & 31, first = j0 + 32 * lane;
-            if (lane < 4 && first < c.q_end)
-                atomicOr(touch + (first >> 5), c.q_end - first >= 32 ? 0xffffffffu : (1u << (c.q_end - first)) - 1u);
-        }
+        TileWalk<kBlock> walk(c);
+        int jt;
+        uint32_t pat;
+        while (walk.next(jt, pat)) {
+            const int j0 = jt * BN;
+            if (a.touch != nullptr) {   // debug: the positions of this tile that exist, 32 per lane 0..3
+                const int lane = threadIdx.x & 31, first = j0 + 32 * lane;
+                if (lane < 4 && first < c.q_end)
+                    atomicOr(a.touch + (first >> 5), c.q_end - first >= 32 ? 0xffffffffu : (1u << (c.q_end - first)) - 1u);
+            }
 #pragma unroll
-        for (int kv = 0; kv < 2; ++kv) {
-            const int qi = 2 * it + kv, slot = qi % kKvSlots, use = qi / kKvSlots;
-            if (!c.wait(BAR_KV_EMPTY + slot, (uint32_t)((use & 1) ^ 1))) return;
-            const uint32_t dst = c.sb + OFF_KV + slot * kTileBytes;
-            const CUtensorMap *tm = kv ? tm_v : tm_k;
-            if (elect_one()) {
-                mbar_expect_tx(c.bar(BAR_KV_FULL + slot), (uint32_t)kTileBytes);
-                tma_load_3d(dst, tm, c.bar(BAR_KV_FULL + slot), 0, c.kvh, j0);
-                tma_load_3d(dst + kHalfBytes, tm, c.bar(BAR_KV_FULL + slot), 64, c.kvh, j0);
+            for (int kv = 0; kv < 2; ++kv, ++qi) {
+                const int slot = qi % kKvSlots, use = qi / kKvSlots;
+                if (!c.wait(BAR_KV_EMPTY + slot, (uint32_t)((use & 1) ^ 1))) return;
+                const uint32_t dst = c.sb + OFF_KV + slot * kTileBytes;
+                const CUtensorMap *tm = kv ? tm_v : tm_k;
+                if (elect_one()) {
+                    mbar_expect_tx(c.bar(BAR_KV_FULL + slot), (uint32_t)kTileBytes);
+                    tma_load_3d(dst, tm, c.bar(BAR_KV_FULL + slot), 0, c.kvh, j0);
+                    tma_load_3d(dst + kHalfBytes, tm, c.bar(BAR_KV_FULL + slot), 64, c.kvh, j0);
+                }
             }
         }
     }
@@ -356,8 +433,11 @@ __device__ __forceinline__ void role_load(const Cta &c, const CUtensorMap *tm_q,
 // Issue order per KV tile j:  PV_0[j] QK_0[j+1] PV_1[j] QK_1[j+1]; the tensor pipe runs them in
 // that order, so S_t[j+1] overwrites S_t / P_t only after PV_t[j] has read P_t[j].  (One issuer for
 // both tiles: two issuing warps, whose MMAs interleave instruction by instruction, ran slower.)
+// Across items the same order holds (the first QK^T of an item follows the last PV of the one
+// before).  The first PV of an item overwrites O_t; it waits for that item's first P_t, which the
+// softmax warps of tile t publish only after their epilogue has read the previous item's O_t.
 template <bool kBlock>
-__device__ __forceinline__ void role_mma(const Cta &c)
+__device__ __forceinline__ void role_mma(Cta &c, const TcArgs &a)
 {
     // S_t = Q_t K^T, then up to two commits (tcgen05.commit belongs to the issuing lane; 0 = none)
     auto qk = [&](int t, int slot, uint32_t bar_a, uint32_t bar_b) {
@@ -387,165 +467,191 @@ __device__ __forceinline__ void role_mma(const Cta &c)
             if (bar_b) tc_commit(bar_b);
         }
     };
-    TileWalk<kBlock> walk(c);
-    int jt;
-    uint32_t pat;
-    bool more = walk.next(jt, pat);
-    if (!c.wait(BAR_Q_FULL, 0)) return;
-    if (!more) {    // (block-mask mode) the item keeps no block at all: nothing to accumulate
-        if (elect_one())
-            for (int t = 0; t < c.nslots; ++t) tc_commit(c.bar(BAR_O_FULL + t));
-        return;
-    }
-    if (!c.wait(BAR_KV_FULL + 0, 0)) return;
-    tc_fence_after();
-    for (int t = 0; t < c.nslots; ++t)
-        qk(t, 0, c.bar(BAR_S_FULL + t), t == c.nslots - 1 ? c.bar(BAR_KV_EMPTY + 0) : 0u);
-    for (int it = 0; more; ++it) {
-        const int vq = 2 * it + 1, vslot = vq % kKvSlots, vpar = (vq / kKvSlots) & 1;
-        const int kq = 2 * it + 2, kslot = kq % kKvSlots, kpar = (kq / kKvSlots) & 1;
-        more = walk.next(jt, pat);
-        if (!c.wait(BAR_KV_FULL + vslot, (uint32_t)vpar)) return;
-        for (int t = 0; t < c.nslots; ++t) {
-            const bool last = t == c.nslots - 1;
-            if (!c.wait(BAR_P_FULL + 2 * t, (uint32_t)(it & 1))) return;
-            tc_fence_after();
-            pv_half(t, vslot, 0, it > 0, 0u, 0u);
-            if (!c.wait(BAR_P_FULL + 2 * t + 1, (uint32_t)(it & 1))) return;
-            tc_fence_after();
-            // after the second half: V slot free once the last tile's PV is done; O complete on the last KV tile
-            pv_half(t, vslot, 1, it > 0, more ? (last ? c.bar(BAR_KV_EMPTY + vslot) : 0u) : c.bar(BAR_O_FULL + t), 0u);
-            if (more) {
-                if (t == 0) {
-                    if (!c.wait(BAR_KV_FULL + kslot, (uint32_t)kpar)) return;
-                    tc_fence_after();
-                }
-                qk(t, kslot, c.bar(BAR_S_FULL + t), last ? c.bar(BAR_KV_EMPTY + kslot) : 0u);
+    int qi = 0;                                      // K / V tiles consumed so far (ring position)
+    int tiles[2] = {0, 0};                           // per query-tile slot: KV tiles done (barrier phases)
+    for (int k = 0;; ++k) {
+        const int item = item_of(k);
+        if (item >= a.n_items) break;
+        decode_item(a, item, c.fa, c);
+        TileWalk<kBlock> walk(c);
+        int jt;
+        uint32_t pat;
+        bool more = walk.next(jt, pat);
+        if (!c.wait(BAR_Q_FULL, (uint32_t)(k & 1))) return;
+        if (!more) {    // (block-mask mode) the item keeps no block at all: nothing to accumulate
+            if (elect_one()) {
+                for (int t = 0; t < c.nslots; ++t) tc_commit(c.bar(BAR_O_FULL + t));
+                tc_commit(c.bar(BAR_Q_EMPTY));
             }
+            continue;
+        }
+        {
+            const int kslot = qi % kKvSlots, kpar = (qi / kKvSlots) & 1;
+            if (!c.wait(BAR_KV_FULL + kslot, (uint32_t)kpar)) return;
+            tc_fence_after();
+            for (int t = 0; t < c.nslots; ++t)
+                qk(t, kslot, c.bar(BAR_S_FULL + t), t == c.nslots - 1 ? c.bar(BAR_KV_EMPTY + kslot) : 0u);
+            ++qi;
+        }
+        for (bool first = true; more; first = false) {
+            const int vslot = qi % kKvSlots, vpar = (qi / kKvSlots) & 1;
+            const int kslot = (qi + 1) % kKvSlots, kpar = ((qi + 1) / kKvSlots) & 1;
+            more = walk.next(jt, pat);
+            if (!c.wait(BAR_KV_FULL + vslot, (uint32_t)vpar)) return;
+            // no QK^T of this item is left to issue once its last tile is reached: Q may be replaced
+            if (!more && elect_one()) tc_commit(c.bar(BAR_Q_EMPTY));
+            for (int t = 0; t < c.nslots; ++t) {
+                const bool last = t == c.nslots - 1;
+                if (!c.wait(BAR_P_FULL + 2 * t, (uint32_t)(tiles[t] & 1))) return;
+                tc_fence_after();
+                pv_half(t, vslot, 0, !first, 0u, 0u);
+                if (!c.wait(BAR_P_FULL + 2 * t + 1, (uint32_t)(tiles[t] & 1))) return;
+                tc_fence_after();
+                // after the second half: the V slot is free once the last tile's PV is done; O is complete on the last KV tile
+                pv_half(t, vslot, 1, !first, last ? c.bar(BAR_KV_EMPTY + vslot) : 0u, more ? 0u : c.bar(BAR_O_FULL + t));
+                tiles[t]++;
+                if (more) {
+                    if (t == 0) {
+                        if (!c.wait(BAR_KV_FULL + kslot, (uint32_t)kpar)) return;
+                        tc_fence_after();
+                    }
+                    qk(t, kslot, c.bar(BAR_S_FULL + t), last ? c.bar(BAR_KV_EMPTY + kslot) : 0u);
+                }
+            }
+            qi += more ? 2 : 1;
         }
     }
 }
 
 // ================= softmax of query tile t (one thread per query row) =================
 template <bool kBlock>
-__device__ __forceinline__ void role_softmax(const Cta &c, const TcArgs &a, int t, int warp, int lane)
+__device__ __forceinline__ void role_softmax(Cta &c, const TcArgs &a, int t, int warp, int lane)
 {
     const int r = (warp & 3) * 32 + lane;            // row of the tile = TMEM lane
-    const int i0 = c.i0(t);                          // first absolute position of this query tile
-    const int row = i0 + r;                          // absolute position of this query
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const uint32_t tS = c.tmem + lane_base + TM_S + t * 128;
     const uint32_t tO = c.tmem + lane_base + TM_O + t * 128;
     const int S = a.S, W = a.W;
     const float scale_log2 = a.scale_log2;
-    float m_used = -INFINITY;                        // running maximum in use, scaled log2 units
-    float2 lsum = make_float2(0.f, 0.f);
-    TileWalk<kBlock> walk(c);
-    int jt;
-    uint32_t pat;
-    for (int it = 0; walk.next(jt, pat); ++it) {
-        if (!c.wait(BAR_S_FULL + t, (uint32_t)(it & 1))) return;
-        tc_fence_after();
-        uint32_t sr[4][32];
+    int tiles = 0, items = 0;                        // KV tiles and items this slot has done (barrier phases)
+    for (int k = 0;; ++k) {
+        const int item = item_of(k);
+        if (item >= a.n_items) break;
+        decode_item(a, item, c.fa, c);
+        if (t >= c.nslots) continue;                 // this item has a single query tile
+        const int i0 = c.i0(t);                      // first absolute position of this query tile
+        const int row = i0 + r;                      // absolute position of this query
+        float m_used = -INFINITY;                    // running maximum in use, scaled log2 units
+        float2 lsum = make_float2(0.f, 0.f);
+        TileWalk<kBlock> walk(c);
+        int jt;
+        uint32_t pat;
+        while (walk.next(jt, pat)) {
+            if (!c.wait(BAR_S_FULL + t, (uint32_t)(tiles & 1))) return;
+            const bool first = walk.it == 1;         // first KV tile of this item: O holds nothing yet
+            ++tiles;
+            tc_fence_after();
+            uint32_t sr[4][32];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) tc_ld32(tS + q * 32, sr[q]);
-        tc_wait_ld();
-        const int j0 = jt * BN;
-        const int jmax = j0 + BN - 1;
-        // this row's two block bits of the tile (block-mask mode): keys [j0, j0+64) and [j0+64, j0+128)
-        const uint32_t mine = pat >> (4 * t + 2 * (r >> 6));
-        const bool full = kBlock ? (jmax <= i0 && ((pat >> (4 * t)) & 0xfu) == 0xfu)
-                                 : ((jmax <= i0) && (c.fa || jmax < S || j0 > i0 + BM - 1 - W));
-        if (!full) {
+            for (int q = 0; q < 4; ++q) tc_ld32(tS + q * 32, sr[q]);
+            tc_wait_ld();
+            const int j0 = jt * BN;
+            const int jmax = j0 + BN - 1;
+            // this row's two block bits of the tile (block-mask mode): keys [j0, j0+64) and [j0+64, j0+128)
+            const uint32_t mine = pat >> (4 * t + 2 * (r >> 6));
+            const bool full = kBlock ? (jmax <= i0 && ((pat >> (4 * t)) & 0xfu) == 0xfu)
+                                     : ((jmax <= i0) && (c.fa || jmax < S || j0 > i0 + BM - 1 - W));
+            if (!full) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const int key = j0 + q * 32 + e;
+                        const bool keep = kBlock ? (key <= row && ((mine >> (q >> 1)) & 1u) != 0u)
+                                                 : (key <= row && (c.fa || key < S || key > row - W));
+                        if (!keep) sr[q][e] = 0xff800000u;   // -inf
+                    }
+            }
+            float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
             for (int q = 0; q < 4; ++q)
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const int key = j0 + q * 32 + e;
-                    const bool keep = kBlock ? (key <= row && ((mine >> (q >> 1)) & 1u) != 0u)
-                                             : (key <= row && (c.fa || key < S || key > row - W));
-                    if (!keep) sr[q][e] = 0xff800000u;   // -inf
+                for (int e = 0; e < 32; e += 2)
+                    mx[q] = fmax3(mx[q], __uint_as_float(sr[q][e]), __uint_as_float(sr[q][e + 1]));
+            const float mxs = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;
+            const bool need = mxs > m_used + kRescaleThreshold;
+            if (__any_sync(0xffffffffu, need)) {
+                const float alpha = need ? fast_exp2(m_used - mxs) : 1.0f;   // 0 when nothing was kept so far
+                if (need) m_used = mxs;
+                lsum.x *= alpha;
+                lsum.y *= alpha;
+                if (!first) {                                                // PV of the previous tile is complete
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t o[32];
+                        tc_ld32(tO + q * 32, o);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+                        tc_st32(tO + q * 32, o);
+                    }
                 }
+            }
+            const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
+            const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(neg_m, neg_m);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t p[32];
+                float2 acc2 = make_float2(0.f, 0.f);
+#pragma unroll
+                for (int qq = 0; qq < 2; ++qq)
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) {
+                        float2 x = ffma2(make_float2(__uint_as_float(sr[2 * half + qq][2 * e]),
+                                                     __uint_as_float(sr[2 * half + qq][2 * e + 1])), sc2, nm2);
+                        x.x = fast_exp2(x.x);
+                        x.y = fast_exp2(x.y);
+                        if (qq == 0) lsum = fadd2(lsum, x); else acc2 = fadd2(acc2, x);
+                        p[16 * qq + e] = pack_bf16(x.x, x.y);
+                    }
+                lsum = fadd2(lsum, acc2);
+                tc_st32(tS + half * 32, p);                  // P columns [32 half, 32 half + 32) = keys [64 half, 64 half + 64)
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(c.bar(BAR_P_FULL + 2 * t + half));
+            }
         }
-        float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+        // ---- epilogue of the item: O / l -> bf16 -> global ----
+        if (!c.wait(BAR_O_FULL + t, (uint32_t)(items & 1))) return;
+        ++items;
+        tc_fence_after();
+        const float lrow = lsum.x + lsum.y;
+        // (block-mask mode) a row whose mask keeps no key: zero output row, flagged
+        const bool empty = kBlock && !(lrow > 0.f);
+        if (empty && row < c.q_end) atomicOr(c.status, FLUX_STATUS_BAD_MASK);
+        const float inv = empty ? 0.f : 1.0f / lrow;
+        const bool valid = row < c.q_end;
+        __nv_bfloat16 *dst = a.out + ((size_t)(valid ? row - a.q_start : 0) * a.Hq + c.head(t)) * kHeadDim;
 #pragma unroll
-        for (int q = 0; q < 4; ++q)
+        for (int q = 0; q < 4; ++q) {
+            uint32_t o[32];
+            tc_ld32(tO + q * 32, o);
+            tc_wait_ld();
+            if (valid) {
 #pragma unroll
-            for (int e = 0; e < 32; e += 2)
-                mx[q] = fmax3(mx[q], __uint_as_float(sr[q][e]), __uint_as_float(sr[q][e + 1]));
-        const float mxs = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;
-        const bool need = mxs > m_used + kRescaleThreshold;
-        if (__any_sync(0xffffffffu, need)) {
-            const float alpha = need ? fast_exp2(m_used - mxs) : 1.0f;   // 0 when nothing was kept so far
-            if (need) m_used = mxs;
-            lsum.x *= alpha;
-            lsum.y *= alpha;
-            if (it > 0) {
+                for (int e = 0; e < 2; ++e) {
+                    uint32_t w[8];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    uint32_t o[32];
-                    tc_ld32(tO + q * 32, o);
-                    tc_wait_ld();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
-                    tc_st32(tO + q * 32, o);
+                    for (int z = 0; z < 8; ++z)
+                        w[z] = empty ? 0u   // O holds nothing meaningful
+                                     : pack_bf16(__uint_as_float(o[16 * e + 2 * z]) * inv, __uint_as_float(o[16 * e + 2 * z + 1]) * inv);
+                    st_global_32B(dst + q * 32 + e * 16, w);
                 }
             }
         }
-        const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used;
-        const float2 sc2 = make_float2(scale_log2, scale_log2), nm2 = make_float2(neg_m, neg_m);
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            uint32_t p[32];
-            float2 acc2 = make_float2(0.f, 0.f);
-#pragma unroll
-            for (int qq = 0; qq < 2; ++qq)
-#pragma unroll
-                for (int e = 0; e < 16; ++e) {
-                    float2 x = ffma2(make_float2(__uint_as_float(sr[2 * half + qq][2 * e]),
-                                                 __uint_as_float(sr[2 * half + qq][2 * e + 1])), sc2, nm2);
-                    x.x = fast_exp2(x.x);
-                    x.y = fast_exp2(x.y);
-                    if (qq == 0) lsum = fadd2(lsum, x); else acc2 = fadd2(acc2, x);
-                    p[16 * qq + e] = pack_bf16(x.x, x.y);
-                }
-            lsum = fadd2(lsum, acc2);
-            tc_st32(tS + half * 32, p);                  // P columns [32 half, 32 half + 32) = keys [64 half, 64 half + 64)
-            tc_wait_st();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(c.bar(BAR_P_FULL + 2 * t + half));
-        }
-    }
-    if (!c.wait(BAR_O_FULL + t, 0)) return;
-    tc_fence_after();
-    const float lrow = lsum.x + lsum.y;
-    // (block-mask mode) a row whose mask keeps no key: zero output row, flagged
-    const bool empty = kBlock && !(lrow > 0.f);
-    if (empty && row < c.q_end) atomicOr(c.status, FLUX_STATUS_BAD_MASK);
-    const float inv = empty ? 0.f : 1.0f / lrow;
-    const bool valid = row < c.q_end;
-    __nv_bfloat16 *dst = a.out + ((size_t)(valid ? row - a.q_start : 0) * a.Hq + c.head(t)) * kHeadDim;
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-        uint32_t o[32];
-        tc_ld32(tO + q * 32, o);
-        tc_wait_ld();
-        if (valid) {
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                uint4 w;
-                if (empty) {
-#pragma unroll
-                    for (int z = 0; z < 8; ++z) o[8 * e + z] = 0u;   // O holds nothing meaningful
-                }
-                w.x = pack_bf16(__uint_as_float(o[8 * e + 0]) * inv, __uint_as_float(o[8 * e + 1]) * inv);
-                w.y = pack_bf16(__uint_as_float(o[8 * e + 2]) * inv, __uint_as_float(o[8 * e + 3]) * inv);
-                w.z = pack_bf16(__uint_as_float(o[8 * e + 4]) * inv, __uint_as_float(o[8 * e + 5]) * inv);
-                w.w = pack_bf16(__uint_as_float(o[8 * e + 6]) * inv, __uint_as_float(o[8 * e + 7]) * inv);
-                *reinterpret_cast<uint4 *>(dst + q * 32 + e * 8) = w;
-            }
-        }
+        // The next item's first P_t is published by these same warps only after this point, and its
+        // first PV (which overwrites O_t) waits for that P_t: O_t needs no hand-over barrier of its own.
     }
 }
 
@@ -571,50 +677,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     __syncthreads();
     if (*c.abort_flag) return;
 
-    // ---- which work item ----
     const int bid = blockIdx.x;
-    // Work items, heaviest (latest query tiles) first.  An item is two query tiles that walk the
-    // same K / V tiles: the same 128 rows of two heads of a KV group, or -- for the head left
-    // over when the group size is odd -- two consecutive row tiles of that head (the earlier
-    // one simply finds its last KV tile fully masked).  Rank r = tiles counted from the end;
-    // ranks come in pairs (2k, 2k+1): n_kv * P head-pair items each, plus n_kv left-over items
-    // (tiles n_qt-1-2k and n_qt-2-2k) listed with the even rank.
-    {
-        const int per2 = a.n_kv * (2 * a.P + a.odd);
-        const int k2 = bid / per2;
-        int rem = bid % per2;
-        int r = 2 * k2;
-        bool leftover = false;
-        if (rem < a.n_kv * a.P) {
-        } else if (rem < a.n_kv * (a.P + a.odd)) {
-            leftover = true;
-            rem -= a.n_kv * a.P;
-        } else {
-            rem -= a.n_kv * (a.P + a.odd);
-            r += 1;
-        }
-        const int qt = a.n_qt - 1 - r;
-        if (!leftover) {
-            c.kvh = rem / a.P;
-            const int pi = rem % a.P;
-            c.head0 = c.kvh * a.G + 2 * pi;
-            c.head1 = c.head0 + 1;
-            c.qt0 = c.qt1 = qt;
-            c.nslots = 2;
-        } else {
-            c.kvh = rem;
-            c.head0 = c.head1 = c.kvh * a.G + a.G - 1;
-            c.qt0 = qt;
-            c.qt1 = qt - 1;
-            c.nslots = qt >= 1 ? 2 : 1;
-        }
-    }
     c.q_end = a.q_start + a.Nq;                           // KV rows present
-    c.i00 = a.q_start + c.qt0 * BM;
-    c.i01 = a.q_start + c.qt1 * BM;
-    const int i0_min = c.nslots == 2 ? c.i01 : c.i00;     // tile 1 is never later than tile 0
-    const int i_hi = min(c.i00 + BM - 1, c.q_end - 1);
-
     const uint8_t mode_raw = kBlock ? (uint8_t)1 : a.mask[a.req * a.L + a.layer];
     if (mode_raw > 1 && tid == 0) atomicOr(a.status, FLUX_STATUS_BAD_MASK);
     c.fa = mode_raw != 0;
@@ -629,17 +693,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
         d[4] = 0; d[5] = two ? a.S : n; d[6] = two ? n - a.W : 0; d[7] = two ? n : 0;
     }
 
-    const int e2 = i_hi / BN + 1;
-    if (c.fa) {
-        c.e1 = 0;
-        c.b2 = 0;
-    } else {
-        c.e1 = min((a.S + BN - 1) / BN, e2);
-        c.b2 = max(c.e1, max(0, i0_min - a.W + 1) / BN);
-    }
-    c.n_tiles = c.e1 + max(0, e2 - c.b2);
-    c.last_tile = e2 - 1;
-
     // ---- set-up: barriers, TMEM ----
     if (tid == 0) {
         mbar_init(c.bar(BAR_Q_FULL), 1);
@@ -653,6 +706,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             mbar_init(c.bar(BAR_P_FULL + 2 * t + 1), 4);
             mbar_init(c.bar(BAR_O_FULL + t), 1);
         }
+        mbar_init(c.bar(BAR_Q_EMPTY), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -670,13 +724,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     if (warp >= 8) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
         if (warp == 8) {
-            role_load<kBlock>(c, &tm_q, &tm_k, &tm_v, a.touch);
+            role_load<kBlock>(c, a, &tm_q, &tm_k, &tm_v);
         } else if (warp == 9) {
-            role_mma<kBlock>(c);
+            role_mma<kBlock>(c, a);
         }
     } else {
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
-        if (warp < 4 * c.nslots) role_softmax<kBlock>(c, a, warp >> 2, warp, lane);
+        role_softmax<kBlock>(c, a, warp >> 2, warp, lane);
     }
 
     // ---- teardown ----
@@ -786,7 +840,8 @@ int launch_prefill_tc(flux_plan *p, int layer, int req, const void *q, const voi
     a.n_kv = c.n_kv_heads;
     a.P = p->G / 2;
     a.odd = p->G & 1;
-    const int n_items = a.n_qt * a.n_kv * a.P + a.odd * a.n_kv * ((a.n_qt + 1) / 2);
+    a.n_items = a.n_qt * a.n_kv * a.P + a.odd * a.n_kv * ((a.n_qt + 1) / 2);
+    const int n_ctas = a.n_items < p->dev.n_sms ? a.n_items : p->dev.n_sms;   // persistent: one CTA per SM
     a.scale_log2 = p->scale_log2;
     a.debug = (int32_t *)(ws + p->lay.debug);
     a.status = (uint32_t *)(ws + p->lay.status);
@@ -795,9 +850,9 @@ int launch_prefill_tc(flux_plan *p, int layer, int req, const void *q, const voi
     a.touch = p->touch;
     const int rec = prof_begin(p, FLUX_KERNEL_PREFILL, st);
     if (block_mask)
-        prefill_tc_kernel<true><<<n_items, kThreads, kSmemBytes, st>>>(tq, tk, tv, a);
+        prefill_tc_kernel<true><<<n_ctas, kThreads, kSmemBytes, st>>>(tq, tk, tv, a);
     else
-        prefill_tc_kernel<false><<<n_items, kThreads, kSmemBytes, st>>>(tq, tk, tv, a);
+        prefill_tc_kernel<false><<<n_ctas, kThreads, kSmemBytes, st>>>(tq, tk, tv, a);
     prof_end(p, rec, st);
     p->launches++;
     if (!block_mask) p->debug_records = 1;
