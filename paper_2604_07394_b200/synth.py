@@ -129,8 +129,26 @@ def fill_normal_bf16_(t: torch.Tensor, seed: int, stream: int) -> torch.Tensor:
 
 # stream ids: tensor kind * 2^12 + layer * 2^6 ... kept simple and collision-free
 def stream_id(kind: str, layer: int = 0, req: int = 0, step: int = 0) -> int:
-    kinds = {"q": 1, "k": 2, "v": 3, "qdec": 4, "kdec": 5, "vdec": 6}
+    kinds = {"q": 1, "k": 2, "v": 3, "qdec": 4, "kdec": 5, "vdec": 6, "router": 7}
     return ((kinds[kind] * 64 + layer) * 64 + req) * 1024 + step
+
+
+def router_weights(seed: int, layer: int, n_features: int, enc_dim: int, head_hidden: int, device="cpu") -> dict:
+    """Random stand-ins for one layer's trained router (Sec. 3.1): bf16 weight matrices with
+    N(0, 1/fan_in) entries and fp32 biases N(0, 0.1^2), so every layer's outputs stay O(1).
+    Keys: w_enc1 [E][F], w_enc2 [E][E], w_head1 [R][E], w_head2 [2][R], b_enc1, b_enc2, b_head1,
+    b_head2.  Drawn on the CPU (the same bits whatever the device) and moved."""
+    shapes = {"w_enc1": (enc_dim, n_features), "w_enc2": (enc_dim, enc_dim),
+              "w_head1": (head_hidden, enc_dim), "w_head2": (2, head_hidden)}
+    out = {}
+    for step, (name, shp) in enumerate(shapes.items()):
+        g = torch.Generator(device="cpu")
+        g.manual_seed(_mix(seed, stream_id("router", layer, 0, step)))
+        w = torch.empty(shp, dtype=torch.float32).normal_(0.0, 1.0, generator=g) / float(np.sqrt(shp[1]))
+        out[name] = w.to(torch.bfloat16).to(device)
+        b = torch.empty(shp[0], dtype=torch.float32).normal_(0.0, 0.1, generator=g)
+        out[name.replace("w_", "b_")] = b.to(device)
+    return out
 
 
 def sample_rows(n_rows_total: int, sink: int, window: int, n_random: int, seed: int,
