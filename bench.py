@@ -268,6 +268,51 @@ def cpu_baseline_decode(db: DecodeBench):
             "parity_max_row_rel": worst}
 
 
+# ---- Layer Router front end (Sec. 3.1): latency per layer -------------------------------------------
+
+def router_frontend_block(flux, dev, peaks, warmup, enc_dim=1024, head_hidden=256):
+    """x_Q segments -> logits for every layer of the cfg2 stack, then the hard decision; the paper
+    quotes 0.20 ms per layer for its router (Sec. 4.3).  Widths are this benchmark's choice (the
+    paper gives none).  Timed with CUDA events over `reps` passes of all layers."""
+    w = synth.WORKLOADS["cfg2"]
+    L, Hq, Hkv = w.n_layers, w.n_q_heads, w.n_kv_heads
+    F = 2 * Hq * D
+    plan = flux.Plan(flux.make_config(L, Hq, Hkv, w.sink, w.window, 1, 4096), dev)
+    q = synth.normal_bf16((4096, Hq, D), w.seed, synth.stream_id("q"), dev)
+    ws = [synth.router_weights(w.seed, l, F, enc_dim, head_hidden, dev) for l in range(L)]
+    logits = torch.zeros((1, L, 2), dtype=torch.float32, device=dev)
+    first, last = q[:100], q[-100:]
+
+    def one_pass():
+        for l in range(L):
+            plan.flux_router_forward(ws[l], first, last, logits[0, l])
+        return plan.flux_router_apply(logits=logits)
+
+    for _ in range(max(3, warmup)):
+        one_pass()
+    torch.cuda.synchronize()
+    reps = 20
+    n0 = plan.flux_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        mask = one_pass()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    assert plan.flux_plan_status() == 0
+    bytes_layer = 2 * (F * enc_dim + enc_dim * enc_dim + enc_dim * head_hidden + 2 * head_hidden) + 2 * 200 * Hq * D
+    return {"workload": "cfg2 stack: 32 layers, x_Q of 32 heads x 128, first 100 + last 100 tokens pooled; "
+                        "encoder width %d, head hidden %d (benchmark's choice)" % (enc_dim, head_hidden),
+            "us_per_layer": ms * 1e3 / L, "ms_all_layers_and_decision": ms,
+            "algorithmic_bytes_per_layer": bytes_layer,
+            "gbs": bytes_layer * L / (ms * 1e-3) / 1e9, "hbm_peak_gbs": peaks["hbm_gbs"],
+            "bound": "launch latency (5 launches per layer, %.1f MB of weights per layer)" % (bytes_layer / 1e6),
+            "gpu_launches": int(plan.flux_launch_count() - n0) // reps,
+            "omega_msr_random_weights": float((mask == 0).float().mean()),
+            "paper_router_ms_per_layer": 0.20}
+
+
 # ---- prefill workload ------------------------------------------------------------------------------
 
 def prefill_block(flux, dev, peaks, warmup):
@@ -684,6 +729,11 @@ def main():
             line["prefill"] = prefill_block(flux, dev, peaks, W_)
         except Exception as e:  # report, never hide
             line["prefill"] = {"error": repr(e)}
+    if not args.no_prefill and world == 1:
+        try:
+            line["router_frontend"] = router_frontend_block(flux, dev, peaks, W_)
+        except Exception as e:  # report, never hide
+            line["router_frontend"] = {"error": repr(e)}
     if not args.no_paper_ratios and world == 1:
         try:
             line["paper_ratios_256k"] = paper_ratio_block(flux, dev, W_)

@@ -87,6 +87,37 @@ int flux_plan_destroy(flux_plan *plan);
 int flux_workspace_size(const flux_config *cfg, size_t *bytes_out);
 int flux_plan_set_workspace(flux_plan *plan, void *workspace /*device*/, size_t bytes);
 
+/* Layer Router front end (Sec. 3.1, "Architecture and Feature Extraction"; Appendix D.1): from
+ * the layer's query tensor x_Q to the routing logits of one (request, layer).
+ *   f  = concat(mean over tokens of q_first, mean over tokens of q_last)      [2*n_q_heads*head_dim]
+ *        (Prefill-Suffix Pooling; index = segment*Hq*D + head*D + channel)
+ *   h1 = silu(w_enc1 f + b_enc1);  u = w_enc2 h1 + b_enc2                      Context Encoder
+ *   h2 = silu(w_head1 u + b_head1); (pi_FA, pi_SA) = w_head2 h2 + b_head2      Router Head
+ * The paper names these stages but not the pooling operator, the widths or the activation; the
+ * token mean and silu(x) = x / (1 + exp(-x)) are this library's choice.
+ *   q_first, q_last  bf16 [n_first][n_q_heads][head_dim] and [n_last][..][..], device: the first
+ *                    and the last prompt tokens of x_Q (the paper pools 100 + 100; shorter
+ *                    prompts pass min(100, n) tokens each, the two may overlap).  n_* >= 1.
+ *   w                host struct of device pointers: weights bf16 row-major [out][in], biases
+ *                    fp32; widths enc_dim (E) and head_hidden (R) multiples of 8, <= 4096;
+ *                    w_enc1 [E][2*Hq*D], w_enc2 [E][E], w_head1 [R][E], w_head2 [2][R] (row 0 = FA).
+ *   logits_out       fp32 [2] on the device, 8-byte aligned, e.g. the (request, layer) slot of the
+ *                    [B][n_layers][2] array later given to flux_router_apply.
+ * Five launches on `stream` (pooling + four matrix-vector products, fp32 accumulation); scratch is
+ * in the workspace, so calls for different layers must be stream-ordered.  Cost does not depend
+ * on the prompt length.  Errors: NULL / misaligned pointers, n_* < 1 -> FLUX_E_INVALID_ARG; widths
+ * not multiples of 8 -> FLUX_E_UNSUPPORTED_SHAPE; widths > 4096 -> FLUX_E_CAPACITY. */
+typedef struct {
+    int32_t enc_dim;       /* E */
+    int32_t head_hidden;   /* R */
+    const void *w_enc1;  const float *b_enc1;
+    const void *w_enc2;  const float *b_enc2;
+    const void *w_head1; const float *b_head1;
+    const void *w_head2; const float *b_head2;
+} flux_router_weights;
+int flux_router_forward(flux_plan *plan, const flux_router_weights *w, const void *q_first, int32_t n_first,
+                        const void *q_last, int32_t n_last, float *logits_out /*device*/, void *stream);
+
 /* Hard routing, once per request batch at prefill; the result is cached for all
  * decode steps (Sec. 3.1 "Deterministic Inference via Hard Routing", Sec. 3.3).
  *   logits       fp32 [B][n_layers][2], FA logit first; device or host memory;

@@ -104,6 +104,7 @@ WorkspaceLayout workspace_layout(const flux_config &c)
     w.host_k = off;       off = align_up(off + B * c.n_kv_heads * kRowBytes, A);
     w.host_v = off;       off = align_up(off + B * c.n_kv_heads * kRowBytes, A);
     w.host_o = off;       off = align_up(off + B * c.n_q_heads * kRowBytes, A);
+    w.router = off;       off = align_up(off + ((size_t)2 * c.n_q_heads * kHeadDim + 3 * kRouterMaxWidth) * sizeof(float), A);
     w.total = off;
     return w;
 }
@@ -399,6 +400,27 @@ int flux_router_apply(flux_plan *plan, const float *logits, const uint8_t *mask_
     plan->d_mask = mask_out;
     plan->mask_B = B;
     return FLUX_OK;
+}
+
+int flux_router_forward(flux_plan *plan, const flux_router_weights *w, const void *q_first, int32_t n_first,
+                        const void *q_last, int32_t n_last, float *logits_out, void *stream)
+{
+    int rc = need_plan(plan, true);
+    if (rc) return rc;
+    if (!w) return fail(FLUX_E_INVALID_ARG, "router weights are NULL");
+    if (!q_first || !q_last || !logits_out) return fail(FLUX_E_INVALID_ARG, "NULL tensor pointer");
+    if (n_first < 1 || n_last < 1) return fail(FLUX_E_INVALID_ARG, "a pooled segment needs at least one token");
+    if (w->enc_dim < 8 || w->head_hidden < 8 || (w->enc_dim & 7) || (w->head_hidden & 7))
+        return fail(FLUX_E_UNSUPPORTED_SHAPE, "router widths %d / %d must be multiples of 8", w->enc_dim, w->head_hidden);
+    if (w->enc_dim > kRouterMaxWidth || w->head_hidden > kRouterMaxWidth)
+        return fail(FLUX_E_CAPACITY, "router widths %d / %d exceed %d", w->enc_dim, w->head_hidden, kRouterMaxWidth);
+    const void *ptrs[] = {w->w_enc1, w->b_enc1, w->w_enc2, w->b_enc2, w->w_head1, w->b_head1, w->w_head2, w->b_head2};
+    for (const void *ptr : ptrs)
+        if (!ptr || !aligned16(ptr)) return fail(FLUX_E_INVALID_ARG, "router weight pointer NULL or not 16-byte aligned");
+    if (!aligned16(q_first) || !aligned16(q_last)) return fail(FLUX_E_INVALID_ARG, "tensor pointers must be 16-byte aligned");
+    if (((uintptr_t)logits_out & 7u) != 0) return fail(FLUX_E_INVALID_ARG, "logits_out must be 8-byte aligned");
+    if (!is_device_ptr(logits_out)) return fail(FLUX_E_INVALID_ARG, "logits_out must be device memory");
+    return launch_router_frontend(plan, w, q_first, n_first, q_last, n_last, logits_out, (cudaStream_t)stream);
 }
 
 int flux_attn_prefill(flux_plan *plan, int32_t layer, int32_t req, const void *q, const void *k,

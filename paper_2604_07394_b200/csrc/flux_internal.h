@@ -20,6 +20,7 @@ constexpr int kDecStages = 3;       // cp.async stages per warp
 constexpr int kDecStageBytes = kDecTile * kRowBytes * 2;  // K tile + V tile
 constexpr int kDecMaxCtas = 512;    // upper bound used to size the workspace
 constexpr int kMaxBatch = 1024;     // prefix tables live in shared memory
+constexpr int kRouterMaxWidth = 4096;   // largest hidden width of the router MLPs (sizes the scratch)
 
 // ---- workspace layout (byte offsets from the workspace base) ----------------
 struct WorkspaceLayout {
@@ -34,6 +35,7 @@ struct WorkspaceLayout {
     size_t host_k;       // bf16  [max_batch][Hkv][D]
     size_t host_v;       // bf16  [max_batch][Hkv][D]
     size_t host_o;       // bf16  [max_batch][Hq][D]
+    size_t router;       // fp32  [2*Hq*D + 3*kRouterMaxWidth] pooled descriptor and hidden activations
     size_t total;
     int64_t slots;
 };
@@ -89,6 +91,9 @@ int check_cuda(cudaError_t e, const char *what);
 // kernel launchers; each returns FLUX_OK or a negative code and bumps plan->launches
 int launch_router(flux_plan *p, const float *d_logits, const uint8_t *d_mask_in, int B,
                   uint8_t *d_mask_out, cudaStream_t st);
+// Layer Router front end: pooled x_Q segments -> encoder -> head -> two logits at d_logits_out
+int launch_router_frontend(flux_plan *p, const flux_router_weights *w, const void *q_first, int n_first,
+                           const void *q_last, int n_last, float *d_logits_out, cudaStream_t st);
 int launch_kv_append(flux_plan *p, int layer, int B, const void *k_new, const void *v_new,
                      void *const *k_caches, void *const *v_caches, const int32_t *pos,
                      cudaStream_t st);

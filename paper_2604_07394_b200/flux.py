@@ -43,7 +43,7 @@ FLUX_KV_COMPACT_SA = 1
 
 EXPORTS = [
     "flux_plan_create", "flux_plan_destroy", "flux_workspace_size", "flux_plan_set_workspace",
-    "flux_router_apply", "flux_attn_prefill", "flux_attn_prefill_blocks", "flux_kv_retain", "flux_kv_append",
+    "flux_router_apply", "flux_router_forward", "flux_attn_prefill", "flux_attn_prefill_blocks", "flux_kv_retain", "flux_kv_append",
     "flux_attn_decode", "flux_attn_decode_step", "flux_attn_decode_noalloc", "flux_attn_decode_host", "flux_attn_prefill_host", "flux_plan_status",
     "flux_debug_dispatch", "flux_debug_touched", "flux_debug_prefill_kernel", "flux_debug_wait_probe", "flux_profile_enable", "flux_profile_read", "flux_launch_count", "flux_last_error", "flux_version",
 ]
@@ -55,6 +55,16 @@ class FluxConfig(ctypes.Structure):
         ("head_dim", ctypes.c_int32), ("sink", ctypes.c_int32), ("window", ctypes.c_int32),
         ("softmax_scale", ctypes.c_float), ("max_batch", ctypes.c_int32),
         ("max_context", ctypes.c_int32), ("kv_layout", ctypes.c_int32),
+    ]
+
+
+class FluxRouterWeights(ctypes.Structure):
+    _fields_ = [
+        ("enc_dim", ctypes.c_int32), ("head_hidden", ctypes.c_int32),
+        ("w_enc1", ctypes.c_void_p), ("b_enc1", ctypes.c_void_p),
+        ("w_enc2", ctypes.c_void_p), ("b_enc2", ctypes.c_void_p),
+        ("w_head1", ctypes.c_void_p), ("b_head1", ctypes.c_void_p),
+        ("w_head2", ctypes.c_void_p), ("b_head2", ctypes.c_void_p),
     ]
 
 
@@ -84,6 +94,7 @@ def load():
     L.flux_workspace_size.argtypes = [cfgp, ctypes.POINTER(sz)]
     L.flux_plan_set_workspace.argtypes = [vp, vp, sz]
     L.flux_router_apply.argtypes = [vp, vp, vp, i32, vp, vp]
+    L.flux_router_forward.argtypes = [vp, ctypes.POINTER(FluxRouterWeights), vp, i32, vp, i32, vp, vp]
     L.flux_attn_prefill.argtypes = [vp, i32, i32, vp, vp, vp, i32, i32, vp, vp]
     L.flux_attn_prefill_blocks.argtypes = [vp, vp, vp, vp, i32, i32, vp, i32, vp, vp]
     L.flux_kv_retain.argtypes = [vp, i32, i32, vp, vp, i32, vp, vp, vp]
@@ -186,6 +197,18 @@ class Plan:
         _check(load().flux_router_apply(self._h, _ptr(logits), _ptr(mask), B, _ptr(mask_out), _stream()))
         self.mask = mask_out          # keep the cached decision alive
         return mask_out
+
+    def flux_router_forward(self, weights, q_first, q_last, logits_out=None):
+        """weights: dict of device tensors (w_enc1, b_enc1, w_enc2, b_enc2, w_head1, b_head1, w_head2,
+        b_head2); q_first / q_last: bf16 [tokens][Hq][D] device tensors; logits_out: fp32 [2] device."""
+        if logits_out is None:
+            logits_out = torch.empty(2, dtype=torch.float32, device=self.device)
+        w = FluxRouterWeights(int(weights["w_enc1"].shape[0]), int(weights["w_head1"].shape[0]),
+                              *[_ptr(weights[k]) for k in ("w_enc1", "b_enc1", "w_enc2", "b_enc2",
+                                                           "w_head1", "b_head1", "w_head2", "b_head2")])
+        _check(load().flux_router_forward(self._h, ctypes.byref(w), _ptr(q_first), int(q_first.shape[0]),
+                                          _ptr(q_last), int(q_last.shape[0]), _ptr(logits_out), _stream()))
+        return logits_out
 
     def flux_attn_prefill(self, layer, req, q, k, v, q_start, out=None):
         Nq = int(q.shape[0])
