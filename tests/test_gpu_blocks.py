@@ -105,3 +105,39 @@ def test_streaming_block_mask_at_32k_sampled_rows(flux, kernel):
     ref = oracle.prefill_blocks(bits(q), bits(k), bits(v), 0, B, bm, SCALE, rr, hh)
     compare(out[torch.from_numpy(rr).to(DEV), torch.from_numpy(hh).to(DEV)], ref, "streaming block mask at 32K")
     assert plan.flux_plan_status() == 0
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (6, 2), (3, 3)])
+def test_sparse_random_mask_with_empty_query_tiles_many_items_per_cta(flux, Hq, Hkv):
+    """8192 tokens give more work items than the GPU has SMs, so CTAs of the tensor-core kernel walk
+    several items each; some 128-row query tiles keep no block at all (their items issue no MMA and
+    must hand the CTA's buffers on cleanly), others keep a sparse random pattern.  Even and odd group
+    sizes (head pairs, left-over heads, plain multi-head attention).  Sampled rows against the oracle;
+    rows of the empty tiles are zero and raise the mask flag."""
+    N = 8192
+    nb = N // B
+    bm = _random_mask(nb, 0.06, 4242 + Hq)
+    empty_tiles = [0, 5, 6, 31, 40, 62, 63]                 # first, adjacent, and the last (heaviest) tiles
+    for t in empty_tiles:
+        bm[2 * t:2 * t + 2, :] = 0
+    bm[2 * 17, :] = 0                                       # half a tile empty: rows 2176..2239
+    plan = flux.Plan(flux.make_config(1, Hq, Hkv, 0, 1, 1, N), DEV)
+    q = synth.normal_bf16((N, Hq, 128), 515, 1, DEV)
+    k = synth.normal_bf16((N, Hkv, 128), 515, 2, DEV)
+    v = synth.normal_bf16((N, Hkv, 128), 515, 3, DEV)
+    out = plan.flux_attn_prefill_blocks(q, k, v, 0, torch.from_numpy(bm).to(DEV))
+    rng = np.random.default_rng(9)
+    rows = np.unique(np.concatenate([rng.integers(0, N, 60), np.array([0, 127, 128, 639, 640, 895, 896, 2175, 2176, 2239, 2240,
+                                                                      3967, 3968, 4095, 4096, 5119, 5120, 7935, 7936, 8191])]))
+    heads = np.arange(Hq, dtype=np.int64)
+    rr = np.repeat(rows, Hq)
+    hh = np.tile(heads, len(rows))
+    ref = oracle.prefill_blocks(bits(q), bits(k), bits(v), 0, B, bm, SCALE, rr, hh)
+    got = out[torch.from_numpy(rr).to(DEV), torch.from_numpy(hh).to(DEV)]
+    kept_any = np.array([bm[r // B].any() for r in rr])     # rows of an empty mask row: exact zeros on both sides
+    assert not ref[~kept_any].any() and torch.count_nonzero(got[torch.from_numpy(~kept_any).to(DEV)]) == 0
+    compare(got[torch.from_numpy(kept_any).to(DEV)], ref[kept_any], "sparse mask with empty tiles")
+    for t in empty_tiles:
+        assert torch.count_nonzero(out[128 * t:128 * t + 128]) == 0
+    assert torch.count_nonzero(out[2176:2240]) == 0 and torch.count_nonzero(out[2240:2304]) > 0
+    assert plan.flux_plan_status(raise_on_flag=False) == flux.FLUX_STATUS_BAD_MASK
