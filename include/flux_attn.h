@@ -204,6 +204,23 @@ int flux_attn_decode_step(flux_plan *plan, int32_t layer, int32_t B, const void 
                           const void *k_new, const void *v_new, void *const *k_caches,
                           void *const *v_caches, const int32_t *ctx_len, void *out, void *stream);
 
+/* Head-level sparsity, the alternative the paper argues against (Sec. 2.3 "Motivational
+ * Observations", Fig. 1(b); Appendix C.3 "Implementation of Sparsity Baselines"): inside ONE layer
+ * some KV heads (with their query-head groups) attend densely and the others keep only sink +
+ * window.  Same arithmetic as flux_attn_decode, but the mode comes per (request, KV head) from
+ * head_mask instead of the cached layer mask, so the routed stack and a head-level stack of the
+ * same KV byte budget can be timed on the same kernel.  The request is walked over its whole
+ * length if any of its heads is dense; warps that own a sparse head read only its sink + window
+ * rows and idle for the rest of the walk, and the dense heads' rows are 256-byte pieces of the
+ * token-major cache rows -- the fragmented access and the intra-layer imbalance the paper describes.
+ *   head_mask  uint8 [B][n_kv_heads] on the device: 1 = dense (Eq. 1), 0 = sink + window (Eq. 2);
+ *              other values set FLUX_STATUS_BAD_MASK and count as dense.
+ *   other arguments as flux_attn_decode; caches must be in the FLUX_KV_FULL layout
+ *   (else FLUX_E_UNSUPPORTED_SHAPE).  No routing call is needed beforehand. */
+int flux_attn_decode_heads(flux_plan *plan, int32_t B, const void *q, const void *const *k_caches,
+                           const void *const *v_caches, const int32_t *ctx_len,
+                           const uint8_t *head_mask /*device*/, void *out, void *stream);
+
 /* Decode step for callers that cannot allocate device memory at all.  (The paper
  * has no counterpart: this is a packaging variant of flux_attn_decode, not part of
  * the method.)  Who needs it: code that runs inside a host program which owns all

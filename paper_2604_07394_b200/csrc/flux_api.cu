@@ -549,6 +549,23 @@ int flux_attn_decode(flux_plan *plan, int32_t layer, int32_t B, const void *q,
     return launch_decode(plan, layer, B, q, k_caches, v_caches, ctx_len, out, (cudaStream_t)stream);
 }
 
+int flux_attn_decode_heads(flux_plan *plan, int32_t B, const void *q, const void *const *k_caches,
+                           const void *const *v_caches, const int32_t *ctx_len, const uint8_t *head_mask,
+                           void *out, void *stream)
+{
+    int rc = need_plan(plan, true);
+    if (rc) return rc;
+    if (B < 1 || B > plan->cfg.max_batch) return fail(FLUX_E_CAPACITY, "B=%d outside [1, %d]", B, plan->cfg.max_batch);
+    if (plan->cfg.kv_layout != FLUX_KV_FULL)
+        return fail(FLUX_E_UNSUPPORTED_SHAPE, "head-level modes need the full cache layout (heads of a layer share its rows)");
+    if (!q || !k_caches || !v_caches || !ctx_len || !head_mask || !out)
+        return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    if (!is_device_ptr(head_mask)) return fail(FLUX_E_INVALID_ARG, "head_mask must be device memory");
+    if (!aligned16(q) || !aligned16(out)) return fail(FLUX_E_INVALID_ARG, "q / out must be 16-byte aligned");
+    return launch_decode(plan, 0, B, q, k_caches, v_caches, ctx_len, out, (cudaStream_t)stream, nullptr, nullptr,
+                         head_mask);
+}
+
 int flux_attn_decode_step(flux_plan *plan, int32_t layer, int32_t B, const void *q, const void *k_new,
                           const void *v_new, void *const *k_caches, void *const *v_caches,
                           const int32_t *ctx_len, void *out, void *stream)

@@ -45,6 +45,9 @@ struct DecArgs {
     const unsigned char *v_new;
     uint32_t *touch;            // debug bitmap of the cache rows read ([B][touch_words]), or NULL
     int touch_words;
+    // head-level comparison mode (flux_attn_decode_heads): uint8 [B][Hkv], 1 = the KV head's group
+    // attends densely, 0 = sink + window; NULL in the routed (layer-level) calls
+    const uint8_t *head_mask;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -161,8 +164,18 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
 
     // ---- schedule: units per request, prefix sum, equal spans -------------------------------
     for (int b = tid; b < a.B; b += blockDim.x) {
-        ReqInfo r = req_info(a.ctx_len[b], a.mask[b * a.L + a.layer], a.S, a.W, a.layout,
-                             a.max_context, a.status);
+        int mode_raw;
+        if (a.head_mask != nullptr) {   // the request is walked over its full length if any head is dense
+            mode_raw = 0;
+            for (int h = 0; h < a.Hkv; ++h) {
+                const int mh = a.head_mask[b * a.Hkv + h];
+                if (mh > 1) atomicOr(a.status, FLUX_STATUS_BAD_MASK);
+                mode_raw |= (mh != 0);
+            }
+        } else {
+            mode_raw = a.mask[b * a.L + a.layer];
+        }
+        ReqInfo r = req_info(a.ctx_len[b], mode_raw, a.S, a.W, a.layout, a.max_context, a.status);
         s_neff[b] = r.n_eff;
         s_split[b] = r.split;
         s_shift[b] = r.shift;
@@ -262,6 +275,20 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
     unsigned char *my_smem = smem + (size_t)warp * kDecStages * kDecStageBytes;
     const uint32_t my_smem_u32 = smem_u32(my_smem);
 
+    // Rows a KV head reads of request b.  Routed calls: the request's values.  Head-level mode: a
+    // sparse head inside a request that is walked densely keeps sink + window (full cache layout),
+    // so its warps run out of rows after the first few tiles of the request and idle.
+    auto head_rows = [&](int b, int head, int &n_eff, int &split, int &shift) {
+        n_eff = s_neff[b];
+        split = s_split[b];
+        shift = s_shift[b];
+        if (a.head_mask != nullptr && n_eff > a.S + a.W && a.head_mask[b * a.Hkv + head] == 0) {
+            shift = n_eff - a.W - a.S;
+            split = a.S;
+            n_eff = a.S + a.W;
+        }
+    };
+
     // loader state
     UnitIt lit = first;
     int l_b = -1;
@@ -275,7 +302,8 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
                 l_k = (const unsigned char *)a.k_caches[l_b];
                 l_v = (const unsigned char *)a.v_caches[l_b];
             }
-            const int n_eff = s_neff[l_b], split = s_split[l_b], shift = s_shift[l_b];
+            int n_eff, split, shift;
+            head_rows(l_b, head, n_eff, split, shift);
             const int newrow = s_newrow[l_b];
             const int v0 = (lit.x * slices + slice) * kDecTile;
             const uint32_t sbase = my_smem_u32 + stage * kDecStageBytes;
@@ -386,12 +414,17 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
             }
         }
 
+        int n_valid = 0;
         if (cur_active) {
+            int n_eff, split, shift;
+            head_rows(cit.b, cit.hg * hpc + hw, n_eff, split, shift);
+            n_valid = n_eff - (cit.x * slices + slice) * kDecTile;  // may be <= 0 for a trailing empty slice
+        }
+        // (head-level mode: a sparse head's warp has nothing to do on most tiles of a dense walk)
+        if (cur_active && (a.head_mask == nullptr || n_valid > 0)) {
             const int stage = t % kDecStages;
             const uint32_t kb = my_smem_u32 + stage * kDecStageBytes;
             const uint32_t vb = kb + kDecTile * kRowBytes;
-            const int v0 = (cit.x * slices + slice) * kDecTile;
-            const int n_valid = s_neff[cit.b] - v0;  // may be <= 0 for a trailing empty slice
 
             // S = Q K^T for 16 keys
             float s[2][4];
@@ -582,7 +615,7 @@ int decode_setup(flux_plan *p)
 
 int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *const *k_caches,
                   const void *const *v_caches, const int32_t *ctx_len, void *out, cudaStream_t st,
-                  const void *k_new, const void *v_new)
+                  const void *k_new, const void *v_new, const uint8_t *head_mask)
 {
     const flux_config &c = p->cfg;
     char *ws = (char *)p->ws;
@@ -605,6 +638,7 @@ int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *con
     a.v_new = (const unsigned char *)v_new;
     a.touch = p->touch;
     a.touch_words = p->touch_words;
+    a.head_mask = head_mask;
     const int rec = prof_begin(p, FLUX_KERNEL_DECODE, st);
     decode_kernel<<<p->dec_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
     prof_end(p, rec, st);
@@ -754,6 +788,7 @@ extern "C" int flux_attn_decode_noalloc(const flux_config *cfg, int32_t layer, i
     a.v_new = nullptr;
     a.touch = nullptr;
     a.touch_words = 0;
+    a.head_mask = nullptr;
     decode_kernel<<<nd->n_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
     rc = check_cuda(cudaGetLastError(), "decode kernel launch");
     if (rc) return rc;

@@ -99,10 +99,12 @@ int launch_kv_append(flux_plan *p, int layer, int B, const void *k_new, const vo
                      cudaStream_t st);
 int launch_kv_retain(flux_plan *p, int layer, int req, const void *k_src, const void *v_src,
                      int n, void *k_cache, void *v_cache, cudaStream_t st);
-// k_new / v_new non-NULL: the launch also appends the newest token (flux_attn_decode_step)
+// k_new / v_new non-NULL: the launch also appends the newest token (flux_attn_decode_step);
+// head_mask non-NULL: per-KV-head modes [B][Hkv] instead of the routed layer mask (flux_attn_decode_heads)
 int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *const *k_caches,
                   const void *const *v_caches, const int32_t *ctx_len, void *out,
-                  cudaStream_t st, const void *k_new = nullptr, const void *v_new = nullptr);
+                  cudaStream_t st, const void *k_new = nullptr, const void *v_new = nullptr,
+                  const uint8_t *head_mask = nullptr);
 int launch_prefill(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v,
                    int q_start, int Nq, void *out, cudaStream_t st);
 // bracket a dominant-kernel launch with events when profiling is on

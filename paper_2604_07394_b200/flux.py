@@ -44,7 +44,7 @@ FLUX_KV_COMPACT_SA = 1
 EXPORTS = [
     "flux_plan_create", "flux_plan_destroy", "flux_workspace_size", "flux_plan_set_workspace",
     "flux_router_apply", "flux_router_forward", "flux_attn_prefill", "flux_attn_prefill_blocks", "flux_kv_retain", "flux_kv_append",
-    "flux_attn_decode", "flux_attn_decode_step", "flux_attn_decode_noalloc", "flux_attn_decode_host", "flux_attn_prefill_host", "flux_plan_status",
+    "flux_attn_decode", "flux_attn_decode_heads", "flux_attn_decode_step", "flux_attn_decode_noalloc", "flux_attn_decode_host", "flux_attn_prefill_host", "flux_plan_status",
     "flux_debug_dispatch", "flux_debug_touched", "flux_debug_prefill_kernel", "flux_debug_wait_probe", "flux_profile_enable", "flux_profile_read", "flux_launch_count", "flux_last_error", "flux_version",
 ]
 
@@ -100,6 +100,7 @@ def load():
     L.flux_kv_retain.argtypes = [vp, i32, i32, vp, vp, i32, vp, vp, vp]
     L.flux_kv_append.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
+    L.flux_attn_decode_heads.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode_noalloc.argtypes = [cfgp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -247,6 +248,14 @@ class Plan:
             out = torch.empty_like(q)
         _check(load().flux_attn_decode(self._h, layer, B, _ptr(q), _ptr(k_caches), _ptr(v_caches),
                                        _ptr(ctx_len), _ptr(out), _stream()))
+        return out
+
+    def flux_attn_decode_heads(self, B, q, k_caches, v_caches, ctx_len, head_mask, out=None):
+        """head_mask: uint8 device tensor [B][Hkv], 1 = dense head group, 0 = sink + window."""
+        if out is None:
+            out = torch.empty_like(q)
+        _check(load().flux_attn_decode_heads(self._h, B, _ptr(q), _ptr(k_caches), _ptr(v_caches),
+                                             _ptr(ctx_len), _ptr(head_mask), _ptr(out), _stream()))
         return out
 
     def flux_attn_decode_step(self, layer, B, q, k_new, v_new, k_caches, v_caches, ctx_len, out=None):
