@@ -468,6 +468,65 @@ def paper_ratio_block(flux, dev, warmup):
     return res
 
 
+# ---- head-level vs layer-level sparsity at the same KV byte budget (Sec. 2.3, Appendix C.3) ----------
+
+def head_level_block(flux, dev, peaks, warmup, n=262144):
+    """The paper's efficiency argument re-measured on this GPU: batch 1, Llama-3-8B attention shapes,
+    sink 128 + window 2048, half of the KV bytes sparse.  Layer-level: half of the layers sparse
+    (one dense layer call + one sparse layer call stand for a pair of layers).  Head-level: in
+    every layer 4 of the 8 KV heads sparse (two such layer calls).  Same required bytes; per-layer
+    attention-decode times, CUDA events, full cache layout for both."""
+    w = synth.WORKLOADS["cfg3"]
+    Hq, Hkv, S, W = w.n_q_heads, w.n_kv_heads, 128, 2048
+    plan = flux.Plan(flux.make_config(2, Hq, Hkv, S, W, 1, n), dev)
+    plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
+    # two cache sets, used alternately, so that no call finds its rows in L2 (a sparse layer's 17 MB would fit)
+    sets = []
+    for i in range(2):
+        k = synth.normal_bf16((n, Hkv, D), w.seed + i, synth.stream_id("k"), dev)
+        v = synth.normal_bf16((n, Hkv, D), w.seed + i, synth.stream_id("v"), dev)
+        sets.append((k, v, flux.pointer_table([k], dev), flux.pointer_table([v], dev)))
+    q = synth.normal_bf16((1, Hq, D), w.seed, synth.stream_id("qdec"), dev)
+    out = torch.empty_like(q)
+    ctx = torch.tensor([n], dtype=torch.int32, device=dev)
+    hm_half = torch.tensor([[1, 0] * (Hkv // 2)], dtype=torch.uint8, device=dev)
+    calls = {
+        "dense_layer": lambda t: plan.flux_attn_decode(0, 1, q, sets[t][2], sets[t][3], ctx, out),
+        "sparse_layer": lambda t: plan.flux_attn_decode(1, 1, q, sets[t][2], sets[t][3], ctx, out),
+        "head_level_layer": lambda t: plan.flux_attn_decode_heads(1, q, sets[t][2], sets[t][3], ctx, hm_half, out),
+    }
+    ms, reps = {}, 30
+    for name, fn in calls.items():
+        for i in range(max(3, warmup)):
+            fn(i & 1)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(reps):
+            fn(i & 1)
+        e1.record()
+        torch.cuda.synchronize()
+        ms[name] = e0.elapsed_time(e1) / reps
+    assert plan.flux_plan_status() == 0
+    plan.close()
+    row = 2 * Hkv * D * 2
+    bytes_dense, bytes_sparse = n * row, (S + W) * row
+    pair_layer = ms["dense_layer"] + ms["sparse_layer"]
+    pair_head = 2 * ms["head_level_layer"]
+    return {"context": n, "sink": S, "window": W, "batch": 1,
+            "ms_dense_layer": ms["dense_layer"], "ms_sparse_layer": ms["sparse_layer"],
+            "ms_head_level_layer": ms["head_level_layer"],
+            "required_bytes_per_layer_pair": bytes_dense + bytes_sparse,
+            "speedup_layer_level": 2 * ms["dense_layer"] / pair_layer,
+            "speedup_head_level": 2 * ms["dense_layer"] / pair_head,
+            "byte_model_speedup": 2 * bytes_dense / (bytes_dense + bytes_sparse),
+            "gbs_layer_level": (bytes_dense + bytes_sparse) / (pair_layer * 1e-3) / 1e9,
+            "gbs_head_level": (bytes_dense + bytes_sparse) / (pair_head * 1e-3) / 1e9,
+            "hbm_peak_gbs": peaks["hbm_gbs"],
+            "paper": "head-level sparsity gives only marginal decode speedups, layer-level close to proportional "
+                     "(Fig. 1(b), one A800 80GB, batch 1)"}
+
+
 # ---- reference arm: the oracle on host cores ----------------------------------------------------
 
 def run_reference(args):
@@ -739,6 +798,10 @@ def main():
             line["paper_ratios_256k"] = paper_ratio_block(flux, dev, W_)
         except Exception as e:  # report, never hide
             line["paper_ratios_256k"] = {"error": repr(e)}
+        try:
+            line["head_level_vs_layer_level_256k"] = head_level_block(flux, dev, peaks, W_)
+        except Exception as e:  # report, never hide
+            line["head_level_vs_layer_level_256k"] = {"error": repr(e)}
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.barrier()
