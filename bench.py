@@ -470,7 +470,7 @@ def paper_ratio_block(flux, dev, warmup):
 
 # ---- head-level vs layer-level sparsity at the same KV byte budget (Sec. 2.3, Appendix C.3) ----------
 
-def head_level_block(flux, dev, peaks, warmup, n=262144):
+def head_level_block(flux, dev, peaks, warmup, n=262144, reps=30):
     """The paper's efficiency argument re-measured on this GPU: batch 1, Llama-3-8B attention shapes,
     sink 128 + window 2048, half of the KV bytes sparse.  Layer-level: half of the layers sparse
     (one dense layer call + one sparse layer call stand for a pair of layers).  Head-level: in
@@ -495,7 +495,7 @@ def head_level_block(flux, dev, peaks, warmup, n=262144):
         "sparse_layer": lambda t: plan.flux_attn_decode(1, 1, q, sets[t][2], sets[t][3], ctx, out),
         "head_level_layer": lambda t: plan.flux_attn_decode_heads(1, q, sets[t][2], sets[t][3], ctx, hm_half, out),
     }
-    ms, reps = {}, 30
+    ms = {}
     for name, fn in calls.items():
         for i in range(max(3, warmup)):
             fn(i & 1)
@@ -606,6 +606,10 @@ def profile_case(flux, dev, which):
         assert db.plan.flux_plan_status() == 0
         print(json.dumps({"profile_case": "decode", "layers": 2, "launch_bytes": db.bytes_step(0) / 2,
                           "cache_gb": db.cache_bytes / 1e9}))
+    elif which == "heads":     # one dense, one sparse and one half-sparse-heads layer call at 256K tokens
+        res = head_level_block(flux, dev, measured_peaks(), 1, reps=1)
+        print(json.dumps({"profile_case": "heads", "launch_order": "each of dense, sparse, head-level: 3 warm-up + 1",
+                          "required_bytes_per_layer_pair": res["required_bytes_per_layer_pair"]}))
     else:                      # the prefill workload at 8192 tokens, one FA and one SA layer
         w = dataclasses.replace(synth.WORKLOADS["cfg2"], n_layers=2, prompt_len=8192)
         N = w.prompt_len
@@ -636,7 +640,7 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-paper-ratios", action="store_true")
-    ap.add_argument("--profile", default=None, choices=["decode", "prefill"],
+    ap.add_argument("--profile", default=None, choices=["decode", "prefill", "heads"],
                     help="run a small case of one kernel with few launches (for ncu captures) and exit")
     args = ap.parse_args()
     if args.impl == "reference":
