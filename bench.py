@@ -745,7 +745,9 @@ def main():
         e2e = {"value": whole_job_throughput(world, w.batch, e2e_steps, e2e_ms), "unit": "tokens/s",
                "h2d_bytes_per_step": db.h2d_bytes(), "d2h_bytes_per_step": db.d2h_bytes(),
                "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
-               "api": "flux_attn_decode_host per layer: pinned host q/k_new/v_new in, host out"}
+               "api": "flux_attn_decode_host per layer: q / k_new / v_new read from pinned host memory by the ingest kernel, "
+                      "the result written to pinned host memory by the combine kernel (every byte crosses the bus once, "
+                      "inside the timed region)"}
 
     # the oracle runs after the timed regions, so that the GPU does not sit idle (and clock down)
     # for seconds right before them

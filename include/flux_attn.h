@@ -248,11 +248,15 @@ int flux_attn_decode_noalloc(const flux_config *cfg, int32_t layer, int32_t B,
                              const int32_t *ctx_len, void *out, uint32_t *status_out,
                              void *stream);
 
-/* The same decode step for callers whose activations live in host memory: copies
- * q, k_new, v_new (host, pinned for speed) to staging in the workspace, appends,
- * attends, and copies the result to out (host).  Asynchronous on `stream` like
- * the rest; the host buffers must stay untouched until the stream is synchronised.
- * The caches, pointer tables, pos and ctx_len stay on the device. */
+/* The same decode step for callers whose activations live in host memory: brings
+ * q, k_new, v_new (host) to the device, appends, attends, and delivers the result
+ * to out (host).  With pinned (page-locked) buffers the kernels read the inputs from
+ * host memory and write the result there directly, each byte crossing the bus once
+ * and no copy operation in the stream (three launches); with pageable buffers the
+ * call stages them through the workspace with four asynchronous copies.
+ * Asynchronous on `stream` like the rest; the host buffers must stay untouched
+ * until the stream is synchronised.  The caches, pointer tables, pos and ctx_len
+ * stay on the device. */
 int flux_attn_decode_host(flux_plan *plan, int32_t layer, int32_t B, const void *q_host,
                           const void *k_new_host, const void *v_new_host,
                           void *const *k_caches, void *const *v_caches, const int32_t *pos,

@@ -123,6 +123,17 @@ static bool is_device_ptr(const void *p)
     return a.type == cudaMemoryTypeDevice || a.type == cudaMemoryTypeManaged;
 }
 
+// device-side address of a pinned (page-locked, mapped) host buffer, or NULL for any other memory
+static const void *mapped_host_ptr(const void *p)
+{
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    return a.type == cudaMemoryTypeHost ? a.devicePointer : nullptr;
+}
+
 static int need_plan(flux_plan *p, bool need_ws)
 {
     if (!p) return fail(FLUX_E_INVALID_ARG, "plan is NULL");
@@ -217,6 +228,35 @@ __global__ void kv_retain_kernel(const uint4 *__restrict__ k_src, const uint4 *_
             k_dst[row * row_u4 + i] = k_src[(int64_t)p * row_u4 + i];
             v_dst[row * row_u4 + i] = v_src[(int64_t)p * row_u4 + i];
         }
+    }
+}
+
+// flux_attn_decode_host with pinned (device-mapped) activations: one launch reads the request's new
+// K, V rows and its query rows straight from host memory, each byte once -- the K, V rows go into
+// the caches like kv_append_kernel does, the query rows into device staging (the decode kernel
+// re-reads them from every CTA, which must not cross the bus).
+__global__ void host_ingest_kernel(const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
+                                   const uint4 *__restrict__ q_host, uint4 *__restrict__ q_stage, int q_u4,
+                                   void *const *__restrict__ k_caches, void *const *__restrict__ v_caches,
+                                   const int32_t *__restrict__ pos, const uint8_t *__restrict__ mask,
+                                   int L, int layer, int row_u4, int S, int W, int layout,
+                                   int max_context, uint32_t *status)
+{
+    const int b = blockIdx.x;
+    for (int i = threadIdx.x; i < q_u4; i += blockDim.x) q_stage[(int64_t)b * q_u4 + i] = q_host[(int64_t)b * q_u4 + i];
+    const int p = pos[b];
+    if (p < 0) return;
+    if (p >= max_context) {
+        if (threadIdx.x == 0) atomicOr(status, FLUX_STATUS_BAD_LENGTH);
+        return;
+    }
+    const bool compact = (layout == FLUX_KV_COMPACT_SA) && (mask[b * L + layer] == 0);
+    const int64_t row = cache_row(p, compact, S, W);
+    uint4 *kd = (uint4 *)k_caches[b] + row * row_u4;
+    uint4 *vd = (uint4 *)v_caches[b] + row * row_u4;
+    for (int i = threadIdx.x; i < row_u4; i += blockDim.x) {
+        kd[i] = k_new[(int64_t)b * row_u4 + i];
+        vd[i] = v_new[(int64_t)b * row_u4 + i];
     }
 }
 
@@ -596,6 +636,23 @@ int flux_attn_decode_host(flux_plan *plan, int32_t layer, int32_t B, const void 
     void *dq = ws + plan->lay.host_q, *dk = ws + plan->lay.host_k, *dv = ws + plan->lay.host_v,
          *dout = ws + plan->lay.host_o;
     const size_t qb = (size_t)B * c.n_q_heads * kRowBytes, kb = (size_t)B * c.n_kv_heads * kRowBytes;
+    // Pinned host buffers are mapped into the device's address space: the kernels then read the
+    // inputs and write the result in place (three launches, no copy operations in between).
+    const void *mq = mapped_host_ptr(q_host), *mk = mapped_host_ptr(k_new_host), *mv = mapped_host_ptr(v_new_host);
+    void *mo = const_cast<void *>(mapped_host_ptr(out_host));
+    if (mq && mk && mv && mo && aligned16(mq) && aligned16(mk) && aligned16(mv) && aligned16(mo)) {
+        const int row_u4 = c.n_kv_heads * kRowBytes / 16;
+        host_ingest_kernel<<<B, 256, 0, st>>>((const uint4 *)mk, (const uint4 *)mv, (const uint4 *)mq, (uint4 *)dq,
+                                              c.n_q_heads * kRowBytes / 16, k_caches, v_caches, pos, plan->d_mask,
+                                              c.n_layers, layer, row_u4, c.sink, c.window, c.kv_layout,
+                                              c.max_context, (uint32_t *)(ws + plan->lay.status));
+        plan->launches++;
+        rc = check_cuda(cudaGetLastError(), "host ingest kernel launch");
+        if (!rc)
+            rc = launch_decode(plan, layer, B, dq, (const void *const *)k_caches, (const void *const *)v_caches,
+                               ctx_len, mo, st);
+        return rc;
+    }
     rc = check_cuda(cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, st), "q upload");
     if (!rc) rc = check_cuda(cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, st), "k upload");
     if (!rc) rc = check_cuda(cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, st), "v upload");

@@ -415,7 +415,9 @@ def test_fused_decode_step_equals_append_then_decode(flux, layout):
     assert plan.flux_plan_status() == 0
 
 
-def test_decode_host_entry_point_matches_device_entry_point(flux):
+@pytest.mark.parametrize("pinned", [True, False], ids=["pinned_zero_copy", "pageable_staged"])
+def test_decode_host_entry_point_matches_device_entry_point(flux, pinned):
+    pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
     Hq, Hkv, S, W, B, L = 8, 2, 4, 8, 3, 2
     lens = [30, 9, 17]
     plan = _plan(flux, L, Hq, Hkv, S, W, B, 64)
@@ -423,12 +425,12 @@ def test_decode_host_entry_point_matches_device_entry_point(flux):
     kc = [synth.normal_bf16((64, Hkv, 128), 5, b, DEV) for b in range(B)]
     vc = [synth.normal_bf16((64, Hkv, 128), 6, b, DEV) for b in range(B)]
     kc2 = [t.clone() for t in kc]; vc2 = [t.clone() for t in vc]
-    q = synth.normal_bf16((B, Hq, 128), 7, 0, "cpu").pin_memory()
-    kn = synth.normal_bf16((B, Hkv, 128), 7, 1, "cpu").pin_memory()
-    vn = synth.normal_bf16((B, Hkv, 128), 7, 2, "cpu").pin_memory()
+    q = pin(synth.normal_bf16((B, Hq, 128), 7, 0, "cpu"))
+    kn = pin(synth.normal_bf16((B, Hkv, 128), 7, 1, "cpu"))
+    vn = pin(synth.normal_bf16((B, Hkv, 128), 7, 2, "cpu"))
     pos = torch.tensor([n - 1 for n in lens], dtype=torch.int32, device=DEV)
     ctx = torch.tensor(lens, dtype=torch.int32, device=DEV)
-    out_h = torch.empty((B, Hq, 128), dtype=torch.bfloat16).pin_memory()
+    out_h = pin(torch.empty((B, Hq, 128), dtype=torch.bfloat16))
     for layer in range(L):
         kt, vt = flux.pointer_table(kc, DEV), flux.pointer_table(vc, DEV)
         plan.flux_attn_decode_host(layer, B, q, kn, vn, kt, vt, pos, ctx, out_h)
