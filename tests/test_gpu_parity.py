@@ -439,3 +439,77 @@ def test_decode_host_entry_point_matches_device_entry_point(flux, pinned):
         plan.flux_kv_append(layer, B, kn.to(DEV), vn.to(DEV), kt2, vt2, pos)
         out_d = plan.flux_attn_decode(layer, B, q.to(DEV), kt2, vt2, ctx)
         assert torch.equal(out_d.cpu(), out_h)
+
+
+def test_decode_at_the_maximum_batch_and_group_size(flux):
+    """The largest batch a plan accepts (1024 requests, ragged tiny contexts, some inactive), in both
+    modes, on shared caches; and the largest group size (16 query heads per KV head).  A sample of
+    the requests is checked against the oracle, inactive requests give zero rows."""
+    B, Hq, Hkv, S, W = 1024, 4, 2, 4, 8
+    rng = np.random.default_rng(1024)
+    lens = rng.integers(0, 41, size=B).astype(np.int32)
+    lens[[0, 1, 2, B - 1]] = [40, 0, 1, 33]
+    mask = rng.integers(0, 2, size=(B, 1)).astype(np.uint8)
+    plan = _plan(flux, 1, Hq, Hkv, S, W, B, 64)
+    plan.flux_router_apply(mask=mask)
+    k = synth.normal_bf16((64, Hkv, 128), 31, 1, DEV)      # every request reads the same cache (own length)
+    v = synth.normal_bf16((64, Hkv, 128), 31, 2, DEV)
+    ktab, vtab = flux.pointer_table([k] * B, DEV), flux.pointer_table([v] * B, DEV)
+    q = synth.normal_bf16((B, Hq, 128), 32, 0, DEV)
+    out = plan.flux_attn_decode(0, B, q, ktab, vtab, torch.from_numpy(lens).to(DEV))
+    kb, vb = bits(k), bits(v)
+    for b in list(range(0, 8)) + list(rng.integers(8, B, 40)) + [B - 1]:
+        n = int(lens[b])
+        if n == 0:
+            assert torch.count_nonzero(out[b]) == 0
+            continue
+        ref = oracle.decode(int(mask[b, 0]), bits(q[b]), kb[:n], vb[:n], n, S, W, _scale())
+        compare(out[b], ref, "max batch decode b=%d n=%d" % (b, n))
+    assert torch.count_nonzero(out[torch.from_numpy(lens == 0).to(DEV)]) == 0
+    assert plan.flux_plan_status() == 0
+    with pytest.raises(flux.FluxError) as e:               # one request more than the plan was made for
+        flux.Plan(flux.make_config(1, Hq, Hkv, S, W, B + 1, 64), DEV)
+    assert e.value.code == flux.FLUX_E_CAPACITY
+
+    # 16 query heads per KV head, prefill and decode
+    Hq, Hkv, S, W, N = 32, 2, 16, 48, 300
+    plan = _plan(flux, 2, Hq, Hkv, S, W, 1, 512)
+    plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
+    qp = synth.normal_bf16((N, Hq, 128), 33, 0, DEV)
+    k = synth.normal_bf16((N, Hkv, 128), 33, 1, DEV)
+    v = synth.normal_bf16((N, Hkv, 128), 33, 2, DEV)
+    ktab, vtab = flux.pointer_table([k], DEV), flux.pointer_table([v], DEV)
+    ctx = torch.tensor([N], dtype=torch.int32, device=DEV)
+    for layer, mode in ((0, oracle.FA), (1, oracle.SA)):
+        compare(plan.flux_attn_prefill(layer, 0, qp, k, v, 0),
+                oracle.prefill(mode, bits(qp), bits(k), bits(v), 0, S, W, _scale()), "G=16 prefill mode %d" % mode)
+        compare(plan.flux_attn_decode(layer, 1, qp[N - 1:N].contiguous(), ktab, vtab, ctx)[0],
+                oracle.decode(mode, bits(qp[N - 1]), bits(k), bits(v), N, S, W, _scale()), "G=16 decode mode %d" % mode)
+    assert plan.flux_plan_status() == 0
+
+
+def test_context_exactly_at_and_beyond_max_context(flux):
+    """ctx_len == max_context is legal (the last cache row is used); max_context + 1 is clamped and
+    flagged by the kernel, and the host refuses a prefill that would pass the end."""
+    Hq, Hkv, S, W, cap = 8, 2, 8, 24, 257
+    plan = _plan(flux, 2, Hq, Hkv, S, W, 2, cap)
+    plan.flux_router_apply(mask=np.array([[1, 0], [0, 1]], dtype=np.uint8))
+    k = synth.normal_bf16((cap, Hkv, 128), 41, 1, DEV)
+    v = synth.normal_bf16((cap, Hkv, 128), 41, 2, DEV)
+    ktab, vtab = flux.pointer_table([k, k], DEV), flux.pointer_table([v, v], DEV)
+    q = synth.normal_bf16((2, Hq, 128), 42, 0, DEV)
+    for layer in (0, 1):
+        out = plan.flux_attn_decode(layer, 2, q, ktab, vtab, torch.tensor([cap, cap - 1], dtype=torch.int32, device=DEV))
+        for b, n in ((0, cap), (1, cap - 1)):
+            mode = int(plan.mask[b, layer])
+            compare(out[b], oracle.decode(mode, bits(q[b]), bits(k), bits(v), n, S, W, _scale()), "ctx at capacity")
+    assert plan.flux_plan_status() == 0
+    plan.flux_attn_decode(0, 2, q, ktab, vtab, torch.tensor([cap + 1, 5], dtype=torch.int32, device=DEV))
+    assert plan.flux_plan_status(raise_on_flag=False) == flux.FLUX_STATUS_BAD_LENGTH
+    qp = synth.normal_bf16((4, Hq, 128), 43, 0, DEV)
+    with pytest.raises(flux.FluxError) as e:
+        plan.flux_attn_prefill(0, 0, qp, k, v, cap - 3)
+    assert e.value.code == flux.FLUX_E_CAPACITY
+    out = plan.flux_attn_prefill(0, 0, qp, k, v, cap - 4)      # the last four positions: fits exactly
+    ref = oracle.prefill(oracle.FA, bits(qp), bits(k), bits(v), cap - 4, S, W, _scale())
+    compare(out, ref, "prefill chunk ending at max_context")
