@@ -509,7 +509,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
 // Merge the partials of one (request, query head) and write the bf16 output row.
 // Split-K combine: m = max m_p, l = sum l_p 2^(m_p - m), O = sum O_p 2^(m_p - m) / l over the
 // partials of one (request, query head).  One CTA per (request, head); its 16 warps take the
-// partials round-robin, four at a time with all loads issued before any is used (at batch 1 one
+// partials round-robin, eight at a time with all loads issued before any is used (at batch 1 one
 // head has a few hundred partials, and a loop of dependent loads would cost more than the decode
 // kernel itself), then the warps' results are merged through shared memory.
 constexpr int kCombWarps = 16;
@@ -541,7 +541,7 @@ __global__ void __launch_bounds__(kCombWarps * 32) decode_combine_kernel(DecArgs
 
     float m = kNegBig, l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    constexpr int kUnroll = 4;
+    constexpr int kUnroll = 8;
     for (int p0 = warp; p0 < n_part; p0 += kCombWarps * kUnroll) {
         float mp[kUnroll], lp[kUnroll];
         float4 op[kUnroll];
