@@ -313,6 +313,7 @@ int flux_profile_read(flux_plan *plan, int32_t kind, double *total_ms, int64_t *
 #define FLUX_PREFILL_AUTO     0
 #define FLUX_PREFILL_WARP_MMA 1
 #define FLUX_PREFILL_TCGEN05  2
+#define FLUX_PREFILL_TCGEN05_PAIR 3  /* CTA pairs sharing K / V tiles; group sizes that are multiples of 4, else as 2 */
 int flux_debug_prefill_kernel(flux_plan *plan, int32_t which);
 
 /* Exercises the give-up path of the kernels' bounded waits without any fault: launches one warp

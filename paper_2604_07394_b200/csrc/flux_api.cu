@@ -527,7 +527,7 @@ int flux_debug_prefill_kernel(flux_plan *plan, int32_t which)
 {
     int rc = need_plan(plan, false);
     if (rc) return rc;
-    if (which < FLUX_PREFILL_AUTO || which > FLUX_PREFILL_TCGEN05)
+    if (which < FLUX_PREFILL_AUTO || which > FLUX_PREFILL_TCGEN05_PAIR)
         return fail(FLUX_E_INVALID_ARG, "unknown prefill kernel selector %d", which);
     plan->prefill_kernel = which;
     return FLUX_OK;

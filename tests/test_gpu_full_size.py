@@ -28,7 +28,7 @@ def _sample_heads(Hq, G):
     return sorted({0, G - 1, G, Hq // 2, Hq - G, Hq - 1} & set(range(Hq)))
 
 
-@pytest.mark.parametrize("cfg,kernel", [("cfg2", 0), ("cfg2", 1), ("cfg4", 0)])
+@pytest.mark.parametrize("cfg,kernel", [("cfg2", 0), ("cfg2", 1), ("cfg2", 3), ("cfg4", 0)])
 def test_prefill_full_size_sampled_rows(flux, cfg, kernel):
     """cfg2: 32K tokens, 32/8 heads, sink 128 + window 2048; cfg4: 128K tokens, 28/4 heads (7 query
     heads per KV head), sink 128 + window 4096.  One FA and one SA layer each, whole prompt in one
