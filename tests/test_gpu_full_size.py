@@ -127,3 +127,47 @@ def test_decode_full_size_sampled(flux, cfg):
             want = oracle.kept(mode, n - 1, S, W).tolist()
             assert (compact_rows_to_positions(rows, n, S, W) if mode == 0 else rows) == want
     assert db.plan.flux_plan_status() == 0
+
+
+def test_sparse_outputs_ignore_keys_outside_the_kept_set_at_full_size(flux):
+    """A property that needs no oracle and holds at any size: changing K and V at positions a query does
+    not keep must leave its output bit-identical.  32K prefill (both tensor-core kernels) and a 64K
+    decode in the full cache layout; the FA layer, which keeps those positions, must change."""
+    w = synth.WORKLOADS["cfg2"]
+    N, Hq, Hkv, S, W = w.prompt_len, w.n_q_heads, w.n_kv_heads, w.sink, w.window
+    plan = flux.Plan(flux.make_config(2, Hq, Hkv, S, W, 1, 65536 + 8), DEV)
+    plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
+    q = synth.normal_bf16((N, Hq, 128), w.seed, synth.stream_id("q"), DEV)
+    k = synth.normal_bf16((N, Hkv, 128), w.seed, synth.stream_id("k"), DEV)
+    v = synth.normal_bf16((N, Hkv, 128), w.seed, synth.stream_id("v"), DEV)
+    a, b = 5000, 6000                                   # positions [a, b) are rewritten
+    k2, v2 = k.clone(), v.clone()
+    k2[a:b] = synth.normal_bf16((b - a, Hkv, 128), 99, 1, DEV)
+    v2[a:b] = synth.normal_bf16((b - a, Hkv, 128), 99, 2, DEV)
+    first_unaffected = b - 1 + W                        # the first query whose window starts after b - 1
+    for kernel in (2, 3):
+        plan.flux_debug_prefill_kernel(kernel)
+        sa0, sa1 = plan.flux_attn_prefill(1, 0, q, k, v, 0), plan.flux_attn_prefill(1, 0, q, k2, v2, 0)
+        assert torch.equal(sa0[:a].view(torch.int16), sa1[:a].view(torch.int16))
+        assert torch.equal(sa0[first_unaffected:].view(torch.int16), sa1[first_unaffected:].view(torch.int16))
+        assert not torch.equal(sa0[a:first_unaffected].view(torch.int16), sa1[a:first_unaffected].view(torch.int16))
+        fa0, fa1 = plan.flux_attn_prefill(0, 0, q, k, v, 0), plan.flux_attn_prefill(0, 0, q, k2, v2, 0)
+        assert torch.equal(fa0[:a].view(torch.int16), fa1[:a].view(torch.int16))
+        changed = (fa0[b:] != fa1[b:]).flatten(1).any(dim=1)
+        assert bool(changed.all())                      # every later FA row sees the rewritten keys
+    # decode at 65536 tokens, full layout: rewrite everything between the sink and the window
+    n = 65536
+    kc = synth.normal_bf16((n, Hkv, 128), 7, 1, DEV)
+    vc = synth.normal_bf16((n, Hkv, 128), 7, 2, DEV)
+    kc2, vc2 = kc.clone(), vc.clone()
+    kc2[S:n - W] = synth.normal_bf16((n - W - S, Hkv, 128), 98, 1, DEV)
+    vc2[S:n - W] = synth.normal_bf16((n - W - S, Hkv, 128), 98, 2, DEV)
+    qd = synth.normal_bf16((1, Hq, 128), 7, 3, DEV)
+    ctx = torch.tensor([n], dtype=torch.int32, device=DEV)
+    outs = []
+    for kk, vv in ((kc, vc), (kc2, vc2)):
+        kt, vt = flux.pointer_table([kk], DEV), flux.pointer_table([vv], DEV)
+        outs.append((plan.flux_attn_decode(1, 1, qd, kt, vt, ctx).clone(), plan.flux_attn_decode(0, 1, qd, kt, vt, ctx).clone()))
+    assert torch.equal(outs[0][0].view(torch.int16), outs[1][0].view(torch.int16))          # SA: identical
+    assert not torch.equal(outs[0][1].view(torch.int16), outs[1][1].view(torch.int16))      # FA: differs
+    assert plan.flux_plan_status() == 0
