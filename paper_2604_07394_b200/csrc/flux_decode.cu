@@ -542,25 +542,33 @@ __global__ void __launch_bounds__(kCombWarps * 32) decode_combine_kernel(DecArgs
     float m = kNegBig, l = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     constexpr int kUnroll = 8;
+    // Partial p of this head sits in the slot of CTA c_first + p / slices, slice p % slices.  slices is a
+    // power of two that divides the warp count, so a warp always meets the same slice and walks the CTAs
+    // with a constant stride: all addressing is 32-bit adds on a base computed once.
+    const int sh = 31 - __clz(slices);
+    const int step_c = kCombWarps >> sh;                                    // CTAs between two partials of a warp
+    const int slot0 = (c_first + seg + (warp >> sh)) * kDecWarps + hw + hpc * (warp & (slices - 1));
+    const float *po = a.part_o + ((size_t)slot0 * a.G + r) * kHeadDim + lane * 4;
+    const float *pm = a.part_ml + ((size_t)slot0 * a.G + r) * 2;
+    const int stride_o = step_c * kDecWarps * a.G * kHeadDim, stride_m = step_c * kDecWarps * a.G * 2;
     for (int p0 = warp; p0 < n_part; p0 += kCombWarps * kUnroll) {
         float mp[kUnroll], lp[kUnroll];
         float4 op[kUnroll];
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) {
-            const int p = p0 + u * kCombWarps;
-            if (p < n_part) {
-                const int c = c_first + p / slices, sl = p % slices;
-                const size_t slot = ((size_t)c + seg) * kDecWarps + (hw + hpc * sl);
-                const float2 ml = *reinterpret_cast<const float2 *>(a.part_ml + (slot * a.G + r) * 2);
+            if (p0 + u * kCombWarps < n_part) {
+                const float2 ml = *reinterpret_cast<const float2 *>(pm + u * stride_m);
                 mp[u] = ml.x;
                 lp[u] = ml.y;
-                op[u] = *reinterpret_cast<const float4 *>(a.part_o + (slot * a.G + r) * kHeadDim + lane * 4);
+                op[u] = *reinterpret_cast<const float4 *>(po + u * stride_o);
             } else {
                 mp[u] = kNegBig;
                 lp[u] = 0.f;
                 op[u] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
+        po += kUnroll * stride_o;
+        pm += kUnroll * stride_m;
         float m_new = m;
 #pragma unroll
         for (int u = 0; u < kUnroll; ++u) m_new = fmaxf(m_new, mp[u]);
