@@ -11,7 +11,7 @@
 // Per CTA the roles are those of the one-CTA kernel (warps 0-3 / 4-7 softmax of query tile
 // 0 / 1, warp 8 TMA producer, warp 9 MMA issuer / TMEM allocation); only the leader's warp 9
 // issues MMAs.  Barriers: the loads of both CTAs complete on the leader's Q_FULL / KV_FULL
-// barriers; the leader's commits are multicast to both CTAs' S_FULL / KV_EMPTY / O_FULL /
+// barriers; the leader's commits arrive on both CTAs' S_FULL / KV_EMPTY / O_FULL /
 // Q_EMPTY barriers; the softmax warps of both CTAs arrive on the leader's P_FULL barriers.
 // Every wait is bounded (status bit, clean exit) as in the one-CTA kernel.
 #include <cuda.h>
@@ -118,11 +118,12 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
     asm volatile("cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
                  ::"r"(dst), "l"(tm), "r"(cluster_bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
-// completion of all MMAs issued so far -> one arrival on the barrier at this offset in both CTAs
+// completion of all MMAs issued so far -> one arrival on the barrier at this offset in each of the two
+// CTAs (two commits: this CTA's barrier and, through its cluster-window address, the peer's)
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"((uint16_t)3) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(map_to_cta(bar, 1)) : "memory");
 }
 __device__ __forceinline__ void tc_mma_ss_pair(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc, uint32_t acc)
 {
