@@ -217,6 +217,55 @@ def test_causal_prefix_matches_step_by_step_decode(mode):
         assert np.array_equal(o, O[i])
 
 
+@pytest.mark.parametrize("mode", [oracle.FA, oracle.SA])
+def test_selected_prefill_rows_address_the_same_rows_as_the_full_prefill(mode):
+    """The row-subset evaluation (the one the full-size sampled checks use) against the whole-chunk
+    prefill, which the brute force above pins: a chunk that starts at q_start > 0, rows out of
+    order, heads repeated and out of order.  Q is indexed by (position - q_start), the output by
+    the sample's own index; both slips (position used as the row, head used as the output index)
+    change the result here.  Also against the pure-Python evaluation directly."""
+    rng = np.random.default_rng(31)
+    N, Hq, Hkv, D, S, W = 29, 6, 2, 4, 3, 5
+    Q, K, V = (_rand_bits(rng, s) for s in [(N, Hq, D), (N, Hkv, D), (N, Hkv, D)])
+    full = oracle.prefill(mode, Q, K, V, 0, S, W, 0.45)
+    q_start = 11
+    rows = np.array([28, 11, 19, 12, 28, 20, 11, 27])
+    heads = np.array([5, 5, 0, 3, 1, 3, 0, 2])
+    got = oracle.prefill_rows(mode, Q[q_start:], K, V, q_start, rows, heads, S, W, 0.45)
+    assert got.shape == (len(rows), D)
+    assert np.array_equal(got, full[rows, heads])
+    assert np.array_equal(got, oracle.prefill(mode, Q[q_start:], K, V, q_start, S, W, 0.45)[rows - q_start, heads])
+    Qf, Kf, Vf = (oracle.bits_to_f64(x) for x in (Q, K, V))
+    for t, (i, h) in enumerate(zip(rows.tolist(), heads.tolist())):
+        idx = [j for j in range(i + 1) if mode == oracle.FA or j < S or j >= i - W + 1]
+        assert np.allclose(got[t], _brute(Qf, Kf, Vf, i, h, Hq // Hkv, idx, 0.45), rtol=0, atol=1e-13)
+    # the rows differ from one another, so an index slip cannot hide behind equal values
+    assert len({got[t].tobytes() for t in range(len(rows))}) == len({(int(i), int(h)) for i, h in zip(rows, heads)})
+
+
+@pytest.mark.parametrize("mode", [oracle.FA, oracle.SA])
+def test_decode_head_subset_equals_those_rows_of_the_full_decode(mode):
+    """decode(heads=[...]) reads head h of q and writes sample t of the output: compare with the
+    all-heads decode (pinned above through the prefill) for an unsorted list with a repeat, and
+    with the pure-Python evaluation."""
+    rng = np.random.default_rng(32)
+    n, Hq, Hkv, D, S, W = 21, 6, 3, 4, 2, 6
+    q = _rand_bits(rng, (Hq, D))
+    K, V = _rand_bits(rng, (n + 3, Hkv, D)), _rand_bits(rng, (n + 3, Hkv, D))
+    full = oracle.decode(mode, q, K, V, n, S, W, 0.6)
+    assert full.shape == (Hq, D) and len({full[h].tobytes() for h in range(Hq)}) == Hq
+    for heads in ([5, 0, 3], [3, 0, 5, 3], [4], list(range(Hq))):
+        got = oracle.decode(mode, q, K, V, n, S, W, 0.6, heads=heads)
+        assert got.shape == (len(heads), D)
+        assert np.array_equal(got, full[heads])
+    Kf, Vf = oracle.bits_to_f64(K), oracle.bits_to_f64(V)
+    qf = oracle.bits_to_f64(q)[None]                 # one "row" at index 0 for the helper
+    idx = [j for j in range(n) if mode == oracle.FA or j < S or j >= n - W]
+    got = oracle.decode(mode, q, K, V, n, S, W, 0.6, heads=[5, 0, 3])
+    for t, h in enumerate([5, 0, 3]):
+        assert np.allclose(got[t], _brute(qf, Kf, Vf, 0, h, Hq // Hkv, idx, 0.6), rtol=0, atol=1e-13)
+
+
 @pytest.mark.parametrize("chunk", [1, 7, 64])
 def test_chunked_prefill_is_invariant(chunk):
     rng = np.random.default_rng(10)
@@ -296,6 +345,20 @@ def test_retained_rows_and_compact_slots():
     for n in range(1, 40):
         a, b = set(oracle.retained(n, S, W).tolist()), set(oracle.retained(n + 1, S, W).tolist())
         assert b - a == {n} and len(a - b) <= 1
+
+
+def test_compact_slot_hand_typed_values():
+    """Slot rule of the compact sparse cache, typed out by hand: sink rows stay in place, the rest go
+    round a ring of W rows that starts at slot S (position S -> slot S, S + W -> slot S again)."""
+    table = {  # (S, W): {position: slot}
+        (4, 6): {0: 0, 3: 3, 4: 4, 5: 5, 9: 9, 10: 4, 11: 5, 15: 9, 16: 4, 21: 9, 22: 4},
+        (0, 3): {0: 0, 1: 1, 2: 2, 3: 0, 4: 1, 7: 1, 300: 0},
+        (2, 1): {0: 0, 1: 1, 2: 2, 3: 2, 99: 2},
+        (128, 4096): {127: 127, 128: 128, 4223: 4223, 4224: 128, 8319: 4223, 8320: 128, 65535: 4095, 131071: 4095},
+    }
+    for (S, W), rows in table.items():
+        for j, want in rows.items():
+            assert oracle.compact_slot(j, S, W) == want, (S, W, j)
 
 
 def test_decode_byte_ratio_matches_paper_speedup():
