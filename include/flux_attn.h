@@ -181,9 +181,9 @@ int flux_kv_append(flux_plan *plan, int32_t layer, int32_t B, const void *k_new,
 
 /* One decode step of one layer for the whole batch: one query row per request at
  * position ctx_len-1 (its K, V already appended).  FA requests stream the whole
- * cache, SA requests only sink + window rows (Appendix C.3, "fetches only the
- * locally required KV"); one launch serves mixed modes, split over all SMs in
- * equal-byte spans, followed by a combine pass.
+ * cache, SA requests only their sink + window rows (Appendix C.3); one launch serves
+ * mixed modes, split over all SMs in equal-byte spans, followed by a combine pass (small
+ * batches: one launch does both, see flux_debug_decode_kernel).
  *   q, out    [B][n_q_heads][head_dim], device.
  *   k_caches, v_caches  device arrays of B device pointers.
  *   ctx_len   int32 [B], device: context length including the new token;
@@ -315,6 +315,31 @@ int flux_profile_read(flux_plan *plan, int32_t kind, double *total_ms, int64_t *
 #define FLUX_PREFILL_TCGEN05  2
 #define FLUX_PREFILL_TCGEN05_PAIR 3  /* CTA pairs sharing K / V tiles; group sizes that are multiples of 4, else as 2 */
 int flux_debug_prefill_kernel(flux_plan *plan, int32_t which);
+
+/* Launch overlap for the single-launch decode kernel (off by default).  With it on, a decode launch
+ * builds its schedule and requests its first K / V tiles while the previous kernel in the stream is
+ * still draining, and waits for that kernel only before it reads the query rows, the newest K / V row
+ * (position ctx_len - 1, from the cache or from k_new / v_new) and before it writes anything.  The
+ * caller promises in return that the kernel enqueued immediately before each decode call on the same
+ * stream does not write: ctx_len, the routing mask, the pointer tables, or cache rows of the layer
+ * being read at positions below ctx_len - 1.  (A decode call of the previous layer, flux_kv_append and
+ * flux_attn_decode_step of any layer, and kernels that only produce q / k_new / v_new all qualify.)
+ * Results are the same either way; the two-launch kernels ignore the setting. */
+int flux_plan_set_launch_overlap(flux_plan *plan, int32_t on);
+
+/* Which kernels flux_attn_decode / flux_attn_decode_step launch.  FLUX_DECODE_AUTO (the default)
+ * runs the single-launch kernel for batches of at most 4 requests (the batch-1 latency setting of
+ * Appendix C.3: one launch does the split-K attention and the merge, the CTA that finishes a
+ * (request, KV head) last merges its partials) and the two-launch pair (split-K kernel + combine
+ * pass) above that; the other two values force one of them.  FLUX_DECODE_SINGLE_LAUNCH is honoured
+ * for batches of at most 8 requests and at most 64 KV heads, otherwise the pair runs.  Both compute
+ * Eq. 1 / Eq. 2 over the same rows.  The single-launch kernel is issued with programmatic stream
+ * serialisation: it starts with a grid-dependency wait, so results never depend on it, and it lets
+ * the next such launch in the stream be set up while it drains. */
+#define FLUX_DECODE_AUTO          0
+#define FLUX_DECODE_TWO_LAUNCH    1
+#define FLUX_DECODE_SINGLE_LAUNCH 2
+int flux_debug_decode_kernel(flux_plan *plan, int32_t which);
 
 /* Exercises the give-up path of the kernels' bounded waits without any fault: launches one warp
  * that waits, with the same bounded wait the prefill kernel uses, on a barrier nothing arrives

@@ -160,7 +160,7 @@ void flux_oracle_prefill_rows(int mode, const uint16_t *Q, const uint16_t *K,
 
 /* ---- block-granular sparse patterns ----------------------------------------
  * The sparse kernels the paper runs select keys in blocks (Appendix D.3: the
- * block size, 64, is "the minimum unit of sparsity"; Sec. 4.1 lists block
+ * block size, 64, is the granularity at which keys are kept or dropped; Sec. 4.1 lists block
  * patterns -- streaming, XAttention's selected blocks -- as the sparse modes).
  * A block mask bm[qb][kb] (row-major, n_kb entries per row) says whether query
  * block qb (positions [qb*B, (qb+1)*B)) attends to key block kb; inside a kept

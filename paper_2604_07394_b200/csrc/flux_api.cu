@@ -105,6 +105,7 @@ WorkspaceLayout workspace_layout(const flux_config &c)
     w.host_v = off;       off = align_up(off + B * c.n_kv_heads * kRowBytes, A);
     w.host_o = off;       off = align_up(off + B * c.n_q_heads * kRowBytes, A);
     w.router = off;       off = align_up(off + ((size_t)2 * c.n_q_heads * kHeadDim + 3 * kRouterMaxWidth) * sizeof(float), A);
+    w.tickets = off;      off = align_up(off + (size_t)kDecFusedMaxBatch * c.n_kv_heads * sizeof(uint32_t), A);
     w.total = off;
     return w;
 }
@@ -363,7 +364,10 @@ int flux_plan_create(const flux_config *cfg, flux_plan **plan)
         return fail(FLUX_E_CUDA, "this library is built for sm_100a only (device is sm_%d0)", cc);
     }
     p->dec_ctas = p->dev.n_sms < kDecMaxCtas ? p->dev.n_sms : kDecMaxCtas;
+    p->decode_kernel = FLUX_DECODE_AUTO;
+    p->launch_overlap = 0;
     rc = decode_setup(p);
+    if (!rc) rc = decode_fused_setup(p);
     if (!rc) rc = prefill_setup(p);
     if (rc) {
         delete p;
@@ -530,6 +534,24 @@ int flux_debug_prefill_kernel(flux_plan *plan, int32_t which)
     if (which < FLUX_PREFILL_AUTO || which > FLUX_PREFILL_TCGEN05_PAIR)
         return fail(FLUX_E_INVALID_ARG, "unknown prefill kernel selector %d", which);
     plan->prefill_kernel = which;
+    return FLUX_OK;
+}
+
+int flux_plan_set_launch_overlap(flux_plan *plan, int32_t on)
+{
+    int rc = need_plan(plan, false);
+    if (rc) return rc;
+    plan->launch_overlap = on ? 1 : 0;
+    return FLUX_OK;
+}
+
+int flux_debug_decode_kernel(flux_plan *plan, int32_t which)
+{
+    int rc = need_plan(plan, false);
+    if (rc) return rc;
+    if (which < FLUX_DECODE_AUTO || which > FLUX_DECODE_SINGLE_LAUNCH)
+        return fail(FLUX_E_INVALID_ARG, "unknown decode kernel selector %d", which);
+    plan->decode_kernel = which;
     return FLUX_OK;
 }
 

@@ -3,7 +3,7 @@
 // One launch serves every request of the batch for one layer.  A request in FA
 // mode streams its whole KV cache (Eq. 1); a request in SA mode streams only the
 // sink rows and the window rows (Eq. 2 with the streaming subset; Appendix C.3:
-// the sparse layer "fetches only the locally required KV").  The kept rows of
+// a sparse layer reads only the rows it keeps).  The kept rows of
 // all requests are laid end to end in units of `slices * kDecTile` tokens and cut
 // into gridDim.x equal spans, so every SM streams the same number of bytes
 // whatever the mix of modes and lengths.  Inside a CTA each warp owns one KV
@@ -19,123 +19,13 @@
 
 #include <mutex>
 
-#include "flux_internal.h"
+#include "flux_decode_common.h"
 
 namespace flux {
+
+int launch_decode_fused(flux_plan *p, const DecArgs &a, cudaStream_t st);   // flux_decode_fused.cu
+
 namespace {
-
-constexpr float kNegBig = -1.0e30f;  // finite stand-in for "no key seen yet"
-
-struct DecArgs {
-    const __nv_bfloat16 *q;
-    const void *const *k_caches;
-    const void *const *v_caches;
-    const int32_t *ctx_len;
-    const uint8_t *mask;
-    int B, L, layer, Hq, Hkv, G, S, W, layout, max_context;
-    float scale_log2;
-    float *part_o;
-    float *part_ml;
-    int32_t *debug;
-    int32_t *sched;
-    uint32_t *status;
-    __nv_bfloat16 *out;
-    // fused append (flux_attn_decode_step): the newest token's K, V rows [B][Hkv][D]; NULL otherwise
-    const unsigned char *k_new;
-    const unsigned char *v_new;
-    uint32_t *touch;            // debug bitmap of the cache rows read ([B][touch_words]), or NULL
-    int touch_words;
-    // head-level comparison mode (flux_attn_decode_heads): uint8 [B][Hkv], 1 = the KV head's group
-    // attends densely, 0 = sink + window; NULL in the routed (layer-level) calls
-    const uint8_t *head_mask;
-};
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p)
-{
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait()
-{
-    asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
-}
-
-__device__ __forceinline__ void ldmatrix_x4(uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3,
-                                            uint32_t addr)
-{
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(addr));
-}
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t &r0, uint32_t &r1, uint32_t &r2,
-                                                  uint32_t &r3, uint32_t addr)
-{
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(addr));
-}
-__device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%0,%1,%2,%3};\n"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
-}
-__device__ __forceinline__ float fast_exp2(float x)
-{
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;\n" : "=f"(y) : "f"(x));
-    return y;
-}
-__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
-{
-    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
-    return *reinterpret_cast<uint32_t *>(&v);
-}
-
-// What one request contributes to this layer's launch.
-struct ReqInfo {
-    int n;       // context length after clamping
-    int mode;    // 1 FA, 0 SA
-    int n_eff;   // rows the kernel reads
-    int split;   // virtual rows >= split are shifted by `shift` (window part of a FULL cache)
-    int shift;
-};
-
-__device__ __forceinline__ ReqInfo req_info(int n_raw, int mode_raw, int S, int W, int layout,
-                                            int max_context, uint32_t *status)
-{
-    ReqInfo r;
-    int n = n_raw;
-    if (n > max_context) {
-        atomicOr(status, FLUX_STATUS_BAD_LENGTH);
-        n = max_context;
-    }
-    if (n < 0) n = 0;
-    if (mode_raw > 1) atomicOr(status, FLUX_STATUS_BAD_MASK);
-    r.n = n;
-    r.mode = mode_raw != 0 ? 1 : 0;
-    r.split = 0x7fffffff;
-    r.shift = 0;
-    if (r.mode == 1 || n <= S + W) {
-        r.n_eff = n;  // SA with sink + window >= n keeps every row
-    } else {
-        r.n_eff = S + W;
-        if (layout == FLUX_KV_FULL) {  // rows [0,S) then rows [n-W, n)
-            r.split = S;
-            r.shift = n - W - S;
-        }  // COMPACT_SA: the S + W slots are exactly the kept rows, in slot order
-    }
-    return r;
-}
 
 // position of the unit a warp is loading or consuming
 struct UnitIt {
@@ -180,20 +70,8 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
         s_split[b] = r.split;
         s_shift[b] = r.shift;
         s_units[b] = (r.n_eff + cta_tok - 1) / cta_tok * n_hg;
-        {   // the newest token sits at position n - 1; in a compact sparse cache that is a ring slot
-            const bool compact = a.layout == FLUX_KV_COMPACT_SA && r.mode == 0;
-            const int pnew = r.n - 1;
-            s_newrow[b] = (a.k_new != nullptr && pnew >= 0)
-                              ? ((compact && pnew >= a.S) ? a.S + (pnew - a.S) % a.W : pnew) : -1;
-        }
-        if (blockIdx.x == 0) {
-            int32_t *d = a.debug + b * 8;
-            d[0] = r.mode; d[1] = a.layer; d[2] = b; d[3] = r.n;
-            d[4] = 0;
-            d[5] = (r.split < r.n_eff) ? r.split : r.n_eff;
-            d[6] = (r.split < r.n_eff) ? r.split + r.shift : 0;
-            d[7] = (r.split < r.n_eff) ? r.n_eff + r.shift : 0;
-        }
+        s_newrow[b] = dec_new_row(r, a.k_new != nullptr, a.S, a.W, a.layout);
+        if (blockIdx.x == 0) dec_write_record(a.debug + b * 8, r, a.layer, b);
     }
     __syncthreads();
     if (warp == 0) {
@@ -393,24 +271,8 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
             const int head = cit.hg * hpc + hw;
             cur_active = head < a.Hkv;
             if (cur_active) {
-#pragma unroll
-                for (int nt = 0; nt < 16; ++nt)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) o[nt][e] = 0.f;
-                m_r[0] = m_r[1] = kNegBig;
-                l_r[0] = l_r[1] = 0.f;
-                const __nv_bfloat16 *qb = a.q + ((size_t)cit.b * a.Hq + (size_t)head * a.G) * kHeadDim;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int row = g + 8 * (e & 1);
-                        const int col = kk * 16 + 2 * t4 + 8 * (e >> 1);
-                        qf[kk][e] = row < a.G
-                                        ? *reinterpret_cast<const uint32_t *>(qb + (size_t)row * kHeadDim + col)
-                                        : 0u;
-                    }
-                }
+                dec_state_reset(o, m_r, l_r);
+                dec_load_q(qf, a.q + ((size_t)cit.b * a.Hq + (size_t)head * a.G) * kHeadDim, a.G, lane);
             }
         }
 
@@ -424,81 +286,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
         if (cur_active && (a.head_mask == nullptr || n_valid > 0)) {
             const int stage = t % kDecStages;
             const uint32_t kb = my_smem_u32 + stage * kDecStageBytes;
-            const uint32_t vb = kb + kDecTile * kRowBytes;
-
-            // S = Q K^T for 16 keys
-            float s[2][4];
-#pragma unroll
-            for (int j = 0; j < 2; ++j)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) s[j][e] = 0.f;
-            {
-                const int mi = lane >> 3, rr = lane & 7;
-                const int key = (mi >> 1) * 8 + rr;
-#pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const int chunk = kk * 2 + (mi & 1);
-                    uint32_t b0, b1, b2, b3;
-                    ldmatrix_x4(b0, b1, b2, b3, kb + key * kRowBytes + ((chunk ^ rr) << 4));
-                    mma_bf16(s[0], qf[kk], b0, b1);
-                    mma_bf16(s[1], qf[kk], b2, b3);
-                }
-            }
-            // scale into the log2 domain, mask the ragged tail
-#pragma unroll
-            for (int j = 0; j < 2; ++j)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int key = j * 8 + 2 * t4 + (e & 1);
-                    s[j][e] = key < n_valid ? s[j][e] * a.scale_log2 : -INFINITY;
-                }
-            // online softmax for rows g and g + 8
-            float alpha[2];
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                float mx = fmaxf(fmaxf(s[0][2 * i], s[0][2 * i + 1]), fmaxf(s[1][2 * i], s[1][2 * i + 1]));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-                const float m_new = fmaxf(m_r[i], mx);
-                alpha[i] = fast_exp2(m_r[i] - m_new);
-                m_r[i] = m_new;
-                float rs = 0.f;
-#pragma unroll
-                for (int j = 0; j < 2; ++j)
-#pragma unroll
-                    for (int e = 0; e < 2; ++e) {
-                        const float p = fast_exp2(s[j][2 * i + e] - m_new);
-                        s[j][2 * i + e] = p;
-                        rs += p;
-                    }
-                l_r[i] = l_r[i] * alpha[i] + rs;
-            }
-            uint32_t pa[4];
-            pa[0] = pack_bf16(s[0][0], s[0][1]);
-            pa[1] = pack_bf16(s[0][2], s[0][3]);
-            pa[2] = pack_bf16(s[1][0], s[1][1]);
-            pa[3] = pack_bf16(s[1][2], s[1][3]);
-            // O = alpha * O + P V
-            {
-                const int mi = lane >> 3, rr = lane & 7;
-                const int key = (mi & 1) * 8 + rr;
-#pragma unroll
-                for (int dt = 0; dt < 8; ++dt) {
-                    const int chunk = dt * 2 + (mi >> 1);
-                    uint32_t b0, b1, b2, b3;
-                    ldmatrix_x4_trans(b0, b1, b2, b3, vb + key * kRowBytes + ((chunk ^ rr) << 4));
-#pragma unroll
-                    for (int h2 = 0; h2 < 2; ++h2) {
-                        float(&acc)[4] = o[2 * dt + h2];
-                        acc[0] *= alpha[0];
-                        acc[1] *= alpha[0];
-                        acc[2] *= alpha[1];
-                        acc[3] *= alpha[1];
-                    }
-                    mma_bf16(o[2 * dt], pa, b0, b1);
-                    mma_bf16(o[2 * dt + 1], pa, b2, b3);
-                }
-            }
+            dec_attend_tile(o, m_r, l_r, qf, kb, kb + kDecTile * kRowBytes, n_valid, a.scale_log2, lane);
         }
         advance(cit);
     }
@@ -647,6 +435,12 @@ int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *con
     a.touch = p->touch;
     a.touch_words = p->touch_words;
     a.head_mask = head_mask;
+    a.tickets = (uint32_t *)(ws + p->lay.tickets);
+    a.overlap = (p->launch_overlap && p->touch == nullptr) ? 1 : 0;   // the debug bitmap is written by the loaders
+    const int fused_max = p->decode_kernel == FLUX_DECODE_SINGLE_LAUNCH ? kDecFusedMaxBatch
+                          : p->decode_kernel == FLUX_DECODE_AUTO        ? kDecFusedAutoBatch : 0;
+    if (head_mask == nullptr && B <= fused_max && c.n_kv_heads <= kDecFusedMaxKvHeads)
+        return launch_decode_fused(p, a, st);
     const int rec = prof_begin(p, FLUX_KERNEL_DECODE, st);
     decode_kernel<<<p->dec_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
     prof_end(p, rec, st);
@@ -797,6 +591,8 @@ extern "C" int flux_attn_decode_noalloc(const flux_config *cfg, int32_t layer, i
     a.touch = nullptr;
     a.touch_words = 0;
     a.head_mask = nullptr;
+    a.tickets = nullptr;
+    a.overlap = 0;
     decode_kernel<<<nd->n_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
     rc = check_cuda(cudaGetLastError(), "decode kernel launch");
     if (rc) return rc;

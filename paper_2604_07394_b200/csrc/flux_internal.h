@@ -20,6 +20,9 @@ constexpr int kDecStages = 3;       // cp.async stages per warp
 constexpr int kDecStageBytes = kDecTile * kRowBytes * 2;  // K tile + V tile
 constexpr int kDecMaxCtas = 512;    // upper bound used to size the workspace
 constexpr int kMaxBatch = 1024;     // prefix tables live in shared memory
+constexpr int kDecFusedMaxBatch = 8;    // largest batch the single-launch decode kernel takes
+constexpr int kDecFusedAutoBatch = 4;   // largest batch it is chosen for by default
+constexpr int kDecFusedMaxKvHeads = 64;
 constexpr int kRouterMaxWidth = 4096;   // largest hidden width of the router MLPs (sizes the scratch)
 
 // ---- workspace layout (byte offsets from the workspace base) ----------------
@@ -36,6 +39,7 @@ struct WorkspaceLayout {
     size_t host_v;       // bf16  [max_batch][Hkv][D]
     size_t host_o;       // bf16  [max_batch][Hq][D]
     size_t router;       // fp32  [2*Hq*D + 3*kRouterMaxWidth] pooled descriptor and hidden activations
+    size_t tickets;      // uint32 [kDecFusedMaxBatch][Hkv] arrival counters of the single-launch decode (zero between launches)
     size_t total;
     int64_t slots;
 };
@@ -76,6 +80,8 @@ struct flux_plan {
     int32_t touch_words;    // 32-bit words per request
     int dec_ctas;
     int prefill_kernel;     // FLUX_PREFILL_*
+    int decode_kernel;      // FLUX_DECODE_*
+    int launch_overlap;     // flux_plan_set_launch_overlap
     // optional per-kernel timing (host-side event pool)
     cudaEvent_t *prof_ev;     // 2 * prof_cap events
     int8_t *prof_kind;
@@ -113,7 +119,8 @@ void prof_end(flux_plan *p, int rec, cudaStream_t st);
 int launch_prefill_blocks(flux_plan *p, const void *q, const void *k, const void *v, int q_start, int Nq,
                           const uint8_t *block_mask, int n_kv_blocks, void *out, cudaStream_t st);
 int launch_wait_probe(flux_plan *p, long long limit_cycles, cudaStream_t st);
-int decode_setup(flux_plan *p);   // one-time attribute setting for the decode kernel
+int decode_setup(flux_plan *p);   // one-time attribute setting for the decode kernels
+int decode_fused_setup(flux_plan *p);
 int prefill_setup(flux_plan *p);
 
 }  // namespace flux

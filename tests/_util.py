@@ -12,12 +12,12 @@ REL_TOL = 1e-2      # every output row: ||gpu - ref||_2 <= REL_TOL * ||ref||_2, 
                     # |gpu - ref| <= REL_TOL * (|ref| + rms(ref row))
 # The elementwise rule is a relative bound with an absolute floor tied to the row's own scale
 # (outputs are averages of N(0,1) values, so many elements are near zero and a bare relative
-# error is unbounded).  Where it comes from: the output is rounded to bf16 (<= 2^-9 |ref|), and
-# the softmax weights are rounded to bf16 before the PV product, which adds independent errors
-# whose sum has a standard deviation of about 1.1e-3 * rms(row); over 10^6..10^8 elements its
-# extremes reach 5..6 sigma = 6..7e-3 * rms(row).  An fp64 model of exactly this arithmetic
-# reproduces the kernels' outputs to 1.3e-4 * rms(row), i.e. the kernels add nothing to it.
-
+# error is unbounded).  Where it comes from: the output is rounded to bf16, and the softmax
+# weights are rounded to bf16 before the PV product, which adds independent errors whose sum has
+# a standard deviation of about 1e-3 * rms(row) with extremes of 5..6 sigma over 10^6..10^8
+# elements.  tests/test_tolerance_model.py evaluates that rounding scheme by itself in fp64 and
+# shows where it sits under each of the three bounds.
+# This is the one comparison rule: the smoke check and the benchmark's oracle leg call compare() too.
 
 def compare(gpu, ref, what=""):
     """gpu: bf16/float tensor or array [..., D]; ref: fp64 array of the same shape."""

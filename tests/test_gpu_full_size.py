@@ -88,8 +88,9 @@ def test_prefill_256k_in_chunks_sampled_rows(flux):
     assert plan.flux_plan_status() == 0
 
 
-@pytest.mark.parametrize("cfg", ["cfg3", "cfg4", "cfg5"])
-def test_decode_full_size_sampled(flux, cfg):
+@pytest.mark.parametrize("cfg,dk", [("cfg3", 0), ("cfg3", 2), ("cfg4", 0), ("cfg4", 1), ("cfg4", 3), ("cfg5", 0)],
+                         ids=["cfg3", "cfg3_single_launch", "cfg4", "cfg4_two_launch", "cfg4_overlap", "cfg5"])
+def test_decode_full_size_sampled(flux, cfg, dk):
     """The decode workloads as bench.py builds them (compact sparse caches, per-request masks,
     ragged lengths for cfg5): two steps; at each, for every request two FA and two SA layers are
     checked against the oracle on sampled heads, and every request's dispatch record on those
@@ -100,6 +101,8 @@ def test_decode_full_size_sampled(flux, cfg):
     if cfg == "cfg4":       # decode phase of the 128K workload: the cache is drawn directly
         w = dataclasses.replace(w, prompt_len=0)
     db = bench.DecodeBench(flux, w, DEV, 4)
+    db.plan.flux_debug_decode_kernel(min(dk, 2))     # 0: the default choice for the batch size; 1 / 2: the other kernel
+    db.plan.flux_plan_set_launch_overlap(dk == 3)    # 3: single launch with launch overlap
     heads = _sample_heads(w.n_q_heads, w.n_q_heads // w.n_kv_heads)
     S, W = w.sink, w.window
     for t in (0, 1):

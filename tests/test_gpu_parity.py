@@ -25,9 +25,21 @@ def _scale(D=128):
     return 1.0 / np.sqrt(D)
 
 
-def _plan(flux, L, Hq, Hkv, S, W, B, max_ctx, layout=0):
+def _plan(flux, L, Hq, Hkv, S, W, B, max_ctx, layout=0, decode_kernel=None):
     cfg = flux.make_config(L, Hq, Hkv, S, W, B, max_ctx, kv_layout=layout)
-    return flux.Plan(cfg, DEV)
+    plan = flux.Plan(cfg, DEV)
+    if decode_kernel is not None:
+        plan.flux_debug_decode_kernel(min(decode_kernel, 2))
+        plan.flux_plan_set_launch_overlap(decode_kernel == 3)
+    return plan
+
+
+# Both decode paths run every decode test: the two-launch pair (split-K kernel + combine pass) and the
+# single-launch kernel (taken for batches of at most 8 requests when forced; larger batches fall back
+# to the pair, so those cases run the pair twice); the single-launch kernel also with launch overlap on
+# (schedule and first tile loads ahead of the grid-dependency wait: the calls these tests make keep the
+# promise that mode asks for).
+DECODE_KERNELS = pytest.mark.parametrize("dk", [1, 2, 3], ids=["two_launch", "single_launch", "single_launch_overlap"])
 
 
 # ---- configuration 1 in full: prefill ---------------------------------------------------------
@@ -56,12 +68,13 @@ def test_cfg1_prefill_every_row(flux):
 
 # ---- configuration 1 in full: prefill -> retain -> 16 decode steps, both cache layouts -------
 
+@DECODE_KERNELS
 @pytest.mark.parametrize("layout", [0, 1])
-def test_cfg1_decode_steps(flux, layout):
+def test_cfg1_decode_steps(flux, layout, dk):
     w = synth.WORKLOADS["cfg1"]
     L, Hq, Hkv, S, W, N, T = w.n_layers, w.n_q_heads, w.n_kv_heads, w.sink, w.window, w.prompt_len, w.decode_steps
     mask = synth.layer_masks(w)
-    plan = _plan(flux, L, Hq, Hkv, S, W, 1, N + T, layout)
+    plan = _plan(flux, L, Hq, Hkv, S, W, 1, N + T, layout, dk)
     plan.flux_router_apply(mask=mask)          # host mask, staged by the library
     assert np.array_equal(plan.mask.cpu().numpy(), mask)
     cap_full = N + T
@@ -190,18 +203,23 @@ DECODE_CASES = [
     (32, 8, 128, 256, [1000, 384, 385, 31], 0),
     (24, 12, 5, 20, [90, 25, 26], 1),
     (16, 16, 32, 64, [200, 97], 0),
+    (28, 4, 16, 48, [20000], 0),                                   # batch 1: every CTA busy, several units each
+    (28, 4, 128, 4096, [20000], 1),
+    (8, 8, 64, 128, [5000, 3, 129, 128, 127, 4097, 1, 700], 1),    # the largest batch the single-launch kernel takes
+    (32, 2, 0, 300, [2500, 2500], 0),                              # 16 query heads per KV head (two merge passes)
 ]
 
 
+@DECODE_KERNELS
 @pytest.mark.parametrize("Hq,Hkv,S,W,lens,layout", DECODE_CASES)
-def test_decode_small_shapes(flux, Hq, Hkv, S, W, lens, layout):
+def test_decode_small_shapes(flux, Hq, Hkv, S, W, lens, layout, dk):
     B = len(lens)
     L = 2
     rng = np.random.default_rng(Hq * 100 + Hkv)
     mask = rng.integers(0, 2, size=(B, L)).astype(np.uint8)
     mask[0] = [1, 0]
     cap = max(lens) + 1
-    plan = _plan(flux, L, Hq, Hkv, S, W, B, cap, layout)
+    plan = _plan(flux, L, Hq, Hkv, S, W, B, cap, layout, dk)
     plan.flux_router_apply(mask=torch.from_numpy(mask).to(DEV))      # device mask
     for layer in range(L):
         kc, vc, klog, vlog = [], [], [], []
@@ -248,8 +266,9 @@ def _bits_set(words):
     return np.nonzero(np.unpackbits(w.view(np.uint8), bitorder="little"))[0].tolist()
 
 
+@DECODE_KERNELS
 @pytest.mark.parametrize("layout", [0, 1])
-def test_decode_reads_exactly_the_kept_rows(flux, layout):
+def test_decode_reads_exactly_the_kept_rows(flux, layout, dk):
     """Every cache row whose K / V the decode kernel loads is recorded in a bitmap; per request the
     set must equal the oracle's kept set (mapped through the ring-slot rule for compact caches)."""
     Hq, Hkv, S, W, L = 8, 2, 16, 48, 2
@@ -257,7 +276,7 @@ def test_decode_reads_exactly_the_kept_rows(flux, layout):
     B = len(lens)
     cap = 1024
     mask = np.array([[1, 0], [0, 1], [0, 0], [0, 1], [1, 0], [0, 0]], dtype=np.uint8)
-    plan = _plan(flux, L, Hq, Hkv, S, W, B, cap, layout)
+    plan = _plan(flux, L, Hq, Hkv, S, W, B, cap, layout, dk)
     plan.flux_router_apply(mask=mask)
     touched = torch.zeros((B, cap // 32), dtype=torch.int32, device=DEV)
     plan.flux_debug_touched(touched)
@@ -384,14 +403,15 @@ def test_host_side_argument_errors_launch_nothing(flux):
     assert plan.flux_plan_status(raise_on_flag=False) == flux.FLUX_STATUS_BAD_LENGTH
 
 
+@DECODE_KERNELS
 @pytest.mark.parametrize("layout", [0, 1])
-def test_fused_decode_step_equals_append_then_decode(flux, layout):
+def test_fused_decode_step_equals_append_then_decode(flux, layout, dk):
     """flux_attn_decode_step must leave the same caches and give the same outputs, bit for bit, as
     flux_kv_append followed by flux_attn_decode -- over several steps, so ring slots wrap."""
     Hq, Hkv, S, W, L = 8, 2, 4, 8, 2
     lens = [30, 9, 17, 0, 13]
     B = len(lens)
-    plan = _plan(flux, L, Hq, Hkv, S, W, B, 64, layout)
+    plan = _plan(flux, L, Hq, Hkv, S, W, B, 64, layout, dk)
     mask = np.array([[1, 0], [0, 0], [1, 1], [0, 1], [0, 1]], dtype=np.uint8)
     plan.flux_router_apply(mask=mask)
     for layer in range(L):
