@@ -33,6 +33,8 @@ constexpr int kFuStageBytes = kDecWarps * kDecStages * kDecStageBytes;
 constexpr int kFuMergeOBytes = kDecWarps * kFuRows * kFuRowStride * (int)sizeof(float);
 constexpr int kFuMergeMlBytes = kDecWarps * kFuRows * 2 * (int)sizeof(float);
 constexpr int kFuSmemBytes = kFuStageBytes + kFuMergeOBytes + kFuMergeMlBytes;
+// partial rows (512 bytes of O and 8 bytes of (m, l) each) the idle stage memory takes for the last CTA's merge
+constexpr int kFuStagedRows = kFuStageBytes / (kHeadDim * 4 + 8);
 
 struct FuIt {
     int u;      // global unit index
@@ -193,7 +195,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
     };
 
 #pragma unroll
-    for (int s = 0; s < kDecStages - 1; ++s) {
+    for (int s = 0; s < kDecStages; ++s) {
         if (s < n_units) {
             issue(s, a.overlap != 0);
             advance(lit);
@@ -278,45 +280,47 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
                 *reinterpret_cast<float4 *>(a.part_o + e * kHeadDim + lane * 4) = acc;
                 if (lane == 0) *reinterpret_cast<float2 *>(a.part_ml + e * 2) = make_float2(m, l);
             }
-            __syncthreads();
+            if (pass + 1 < passes) __syncthreads();   // the buffer is reused; after the last pass the ticket barrier does it
         }
-        // release: the CTA's partial stores (ordered before thread 0 by the barrier above) become visible
-        // before the ticket; acquire: the last ticket is followed by a fence before anybody reads partials
+        // One release-acquire ticket per CTA: the CTA's partial stores (ordered before thread 0 by the barrier)
+        // become visible before the ticket is, and whoever draws the last ticket sees every partial.
+        __syncthreads();
         if (tid == 0) {
-            __threadfence();
-            const unsigned ticket = atomicAdd(a.tickets + cur_seg, 1u);
-            __threadfence();
+            unsigned ticket;
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;\n" : "=r"(ticket) : "l"(a.tickets + cur_seg) : "memory");
             s_ticket = ticket;
         }
         __syncthreads();
         if (s_ticket != (unsigned)(n_part - 1)) return;
         // ---- last CTA of the segment ----------------------------------------------------------------
-        // The segment's partials are one contiguous block: entries (c_first + cur_seg) * G ... of n_part * G rows.
+        // The segment's partials are one contiguous block: n_part * G rows from entry (c_first + cur_seg) * G.
         const size_t e_base = ((size_t)c_first + cur_seg) * a.G;
         const int n_rows = n_part * a.G;
-        float2 *s_ml = reinterpret_cast<float2 *>(mo);          // the merge buffer is free now
-        const int cap = idle ? min(kFuStageBytes / (kHeadDim * 4), kFuMergeOBytes / 8) : 0;
-        if (n_rows <= cap) {
-            // all partial rows into the (idle) stage memory with one round of asynchronous copies
+        float2 *s_ml = reinterpret_cast<float2 *>(mml);
+        const float *so = reinterpret_cast<const float *>(smem);
+        if (idle && n_rows <= kFuStagedRows) {
+            // No tile loads are in flight (the CTA's last segment): the block comes into the stage memory by one
+            // round of asynchronous copies; then one warp per query head: weights 2^(m_p - m) first (lanes over
+            // the partials), then the weighted sum with four partials in flight.  The loops stay rolled: this
+            // code runs once per launch, and its size costs more than its arithmetic.
+            float2 *st_ml = reinterpret_cast<float2 *>(smem + (size_t)kFuStagedRows * kHeadDim * 4);
             const unsigned char *src = reinterpret_cast<const unsigned char *>(a.part_o + e_base * kHeadDim);
             const uint32_t dst = smem_u32(smem);
             for (int c = tid; c < n_rows * (kHeadDim * 4 / 16); c += blockDim.x) cp_async16(dst + c * 16, src + (size_t)c * 16, 16);
             cp_async_commit();
-            for (int i = tid; i < n_rows; i += blockDim.x) s_ml[i] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + (e_base + i) * 2));
+            for (int i = tid; i < n_rows; i += blockDim.x) st_ml[i] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + (e_base + i) * 2));
             cp_async_wait<0>();
             __syncthreads();
-            const float *so = reinterpret_cast<const float *>(smem);
             for (int r = warp; r < a.G; r += kDecWarps) {
-                // weights first (lanes over the partials), then the weighted sum with four partials in flight
                 float m = kNegBig;
-                for (int p = lane; p < n_part; p += 32) m = fmaxf(m, s_ml[p * a.G + r].x);
+                for (int p = lane; p < n_part; p += 32) m = fmaxf(m, st_ml[p * a.G + r].x);
 #pragma unroll
                 for (int d = 16; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
                 float l = 0.f;
                 for (int p = lane; p < n_part; p += 32) {
-                    const float2 ml = s_ml[p * a.G + r];
+                    const float2 ml = st_ml[p * a.G + r];
                     const float w = fast_exp2(ml.x - m);
-                    s_ml[p * a.G + r].x = w;
+                    st_ml[p * a.G + r].x = w;
                     l += ml.y * w;
                 }
 #pragma unroll
@@ -326,11 +330,13 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
 #pragma unroll
                 for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
                 const float *row0 = so + (size_t)r * kHeadDim + lane * 4;
+                const float2 *w0 = st_ml + r;
                 int p = 0;
+#pragma unroll 1
                 for (; p + 4 <= n_part; p += 4) {
 #pragma unroll
                     for (int u = 0; u < 4; ++u) {
-                        const float w = s_ml[(p + u) * a.G + r].x;
+                        const float w = w0[(p + u) * a.G].x;
                         const float4 v = *reinterpret_cast<const float4 *>(row0 + (size_t)(p + u) * a.G * kHeadDim);
                         acc[u].x += v.x * w;
                         acc[u].y += v.y * w;
@@ -338,8 +344,9 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
                         acc[u].w += v.w * w;
                     }
                 }
+#pragma unroll 1
                 for (; p < n_part; ++p) {
-                    const float w = s_ml[p * a.G + r].x;
+                    const float w = w0[p * a.G].x;
                     const float4 v = *reinterpret_cast<const float4 *>(row0 + (size_t)p * a.G * kHeadDim);
                     acc[0].x += v.x * w;
                     acc[0].y += v.y * w;
@@ -353,9 +360,9 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
                 *reinterpret_cast<uint2 *>(a.out + ((size_t)seg_b * a.Hq + (size_t)seg_head * a.G + r) * kHeadDim + lane * 4) = pk;
             }
         } else {
-            // tile loads of the next segment are in flight (or the block is too large for the stage memory):
-            // warp w takes partials w, w + 8, ... for every query head straight from global memory, then the
-            // eight warps' results are merged like the per-CTA states above
+            // Tile loads of the next segment are in flight (or the block is too large for the stage memory): warp w
+            // folds partials w, w + 8, ... for every query head straight from global memory, then the eight warps'
+            // results are merged like the per-CTA states above.
             for (int pass = 0; pass < passes; ++pass) {
                 const int rows = min(a.G - pass * kFuRows, kFuRows);
                 float4 acc[kFuRows];
@@ -366,6 +373,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
                     mm[r] = kNegBig;
                     ll[r] = 0.f;
                 }
+#pragma unroll 1
                 for (int p = warp; p < n_part; p += kDecWarps) {
                     const size_t e0 = e_base + (size_t)p * a.G + pass * kFuRows;
                     float2 ml[kFuRows];
@@ -383,19 +391,19 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
 #pragma unroll
                     for (int r = 0; r < kFuRows; ++r) {
                         const float m_new = fmaxf(mm[r], ml[r].x);
-                        const float so = fast_exp2(mm[r] - m_new), sp = fast_exp2(ml[r].x - m_new);
-                        acc[r].x = acc[r].x * so + v[r].x * sp;
-                        acc[r].y = acc[r].y * so + v[r].y * sp;
-                        acc[r].z = acc[r].z * so + v[r].z * sp;
-                        acc[r].w = acc[r].w * so + v[r].w * sp;
-                        ll[r] = ll[r] * so + ml[r].y * sp;
+                        const float sc = fast_exp2(mm[r] - m_new), sp = fast_exp2(ml[r].x - m_new);
+                        acc[r].x = acc[r].x * sc + v[r].x * sp;
+                        acc[r].y = acc[r].y * sc + v[r].y * sp;
+                        acc[r].z = acc[r].z * sc + v[r].z * sp;
+                        acc[r].w = acc[r].w * sc + v[r].w * sp;
+                        ll[r] = ll[r] * sc + ml[r].y * sp;
                         mm[r] = m_new;
                     }
                 }
 #pragma unroll
                 for (int r = 0; r < kFuRows; ++r) {
                     *reinterpret_cast<float4 *>(mo + (warp * kFuRows + r) * kFuRowStride + lane * 4) = acc[r];
-                    if (lane == 0) *reinterpret_cast<float2 *>(mml + (warp * kFuRows + r) * 2) = make_float2(mm[r], ll[r]);
+                    if (lane == 0) s_ml[warp * kFuRows + r] = make_float2(mm[r], ll[r]);
                 }
                 __syncthreads();
                 if (warp < rows) {
@@ -446,7 +454,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
     // the newest row of the tiles that were requested before the wait
     if (patch != 0) {
         FuIt pit = first;
-        for (int st = 0; st < kDecStages - 1 && st < n_units; ++st) {
+        for (int st = 0; st < kDecStages && st < n_units; ++st) {
             const int b = pit.b, head = pit.head;
             const int v0 = pit.x * kFuCtaTok + warp * kDecTile;
 #pragma unroll
@@ -476,16 +484,11 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
     __syncwarp();
     q_fragments();
 
+    // Three tiles are on their way before the first is used; tile t + 3 is requested into the slot of tile t
+    // once that has been consumed.
     for (int t = 0; t < n_units; ++t) {
-        cp_async_wait<kDecStages - 2>();
+        cp_async_wait<kDecStages - 1>();
         __syncwarp();
-        if (t + kDecStages - 1 < n_units) {
-            issue((t + kDecStages - 1) % kDecStages, false);
-            advance(lit);
-        } else {
-            cp_async_commit();
-        }
-
         if (cit.b * a.Hkv + cit.head != cur_seg) {
             flush(false);
             enter_segment(cit);
@@ -497,6 +500,13 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
         const uint32_t kb = my_smem_u32 + (t % kDecStages) * kDecStageBytes;
         dec_attend_tile(o, m_r, l_r, qf, kb, kb + kDecTile * kRowBytes, n_valid, a.scale_log2, lane);
         advance(cit);
+        __syncwarp();
+        if (t + kDecStages < n_units) {
+            issue(t % kDecStages, false);
+            advance(lit);
+        } else {
+            cp_async_commit();
+        }
     }
     cp_async_wait<0>();
     __syncthreads();   // every warp is done with its stage memory
