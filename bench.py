@@ -266,6 +266,74 @@ def cpu_baseline_decode(db: DecodeBench):
             "parity_max_row_rel": worst}
 
 
+def timed_replays(db, steps):
+    """`steps` graph replays bracketed by CUDA events on the current stream -> milliseconds."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        db.step_graph()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def kernel_roofline(db, flux, t, steps, peaks, kernel_name):
+    """The dominant decode kernel, event-bracketed launch by launch on `steps` steps issued call by call."""
+    w = db.w
+    db.plan.flux_profile_enable(steps * w.n_layers + 8)
+    for i in range(steps):
+        db.step(t + i)
+    torch.cuda.synchronize()
+    kms, kcnt = db.plan.flux_profile_read(flux.FLUX_KERNEL_DECODE)
+    db.plan.flux_profile_enable(0)
+    by = sum(db.bytes_step(t + i) for i in range(steps)) / max(kcnt, 1)
+    ms = kms / max(kcnt, 1)
+    ach = by / (ms * 1e-3) / 1e9
+    return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+            "peak_source": peaks["source"] + " (copy bandwidth)", "kernel": kernel_name, "launches_timed": int(kcnt),
+            "avg_launch_ms": ms, "algorithmic_bytes_per_launch": by}
+
+
+def decode_kernel_name(flux, plan_choice, batch):
+    single = plan_choice == "single_launch" and batch <= 8 or plan_choice == "auto" and batch <= 4
+    return ("decode_fused_kernel (split-K decode and merge in one launch per layer)" if single else
+            "decode_kernel (mixed FA/SA split-K decode, one launch per layer)")
+
+
+def secondary_decode_block(flux, dev, peaks, name, steps, warmup, args):
+    """Another decode workload, device-resident: graph replays of the whole step, required bytes / time
+    against the measured HBM copy bandwidth, and its dominant kernel launch by launch."""
+    import dataclasses
+    w = synth.WORKLOADS[name]
+    if w.prompt_len:                       # the decode phase of a prefill + decode workload: the cache is drawn directly
+        w = dataclasses.replace(w, prompt_len=0)
+    roof_steps = 5
+    db = DecodeBench(flux, w, dev, 1 + 2 * warmup + steps + roof_steps + 2, host_mirrors=False)
+    db.plan.flux_debug_decode_kernel({"auto": flux.FLUX_DECODE_AUTO, "two_launch": flux.FLUX_DECODE_TWO_LAUNCH,
+                                      "single_launch": flux.FLUX_DECODE_SINGLE_LAUNCH}[args.decode_kernel])
+    db.plan.flux_plan_set_launch_overlap(not args.no_launch_overlap)
+    t = 0
+    for _ in range(warmup):
+        db.step(t); t += 1
+    n0 = db.plan.flux_launch_count()
+    db.capture_step(t)
+    per_step = db.plan.flux_launch_count() - n0
+    timed_replays(db, warmup); t += warmup
+    t_first = t
+    ms = timed_replays(db, steps); t += steps
+    by = sum(db.bytes_step(i) for i in range(t_first, t_first + steps))
+    roof = kernel_roofline(db, flux, t, roof_steps, peaks, decode_kernel_name(flux, args.decode_kernel, w.batch))
+    assert db.plan.flux_plan_status() == 0
+    gbs = by / (ms * 1e-3) / 1e9
+    res = {"workload": workload_config(w, db.mask, db.ctx0)["workload"], "tokens_per_s": w.batch * steps / (ms * 1e-3),
+           "ms_per_step": ms / steps, "steps": steps, "required_bytes_per_step": by / steps,
+           "step_level_gbs": gbs, "step_level_frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+           "gpu_launches_per_step": int(per_step), "omega_msr": float((db.mask == 0).mean()), "roofline": roof}
+    del db
+    torch.cuda.empty_cache()
+    return res
+
+
 # ---- Layer Router front end (Sec. 3.1): latency per layer -------------------------------------------
 
 def router_frontend_block(flux, dev, peaks, warmup, enc_dim=1024, head_hidden=256):
@@ -394,6 +462,45 @@ def prefill_block(flux, dev, peaks, warmup):
                            "kernel": "FA prefill layer", "traffic": traffic_note("prefill_fa")}
     plan.close()
     return res
+
+
+def prefill_128k_block(flux, dev, peaks, warmup):
+    """One FA and one SA layer of the 128K-token prefill (28 query / 4 KV heads: an odd group of 7, which
+    leaves one head per KV group to the two-row-tiles item shape), each timed alone."""
+    w = synth.WORKLOADS["cfg4"]
+    N, Hq, Hkv, S, W = w.prompt_len, w.n_q_heads, w.n_kv_heads, w.sink, w.window
+    plan = flux.Plan(flux.make_config(2, Hq, Hkv, S, W, 1, N), dev)
+    plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
+    q = synth.normal_bf16((N, Hq, D), w.seed, synth.stream_id("q"), dev)
+    k = synth.normal_bf16((N, Hkv, D), w.seed, synth.stream_id("k"), dev)
+    v = synth.normal_bf16((N, Hkv, D), w.seed, synth.stream_id("v"), dev)
+    out = torch.empty_like(q)
+    i = np.arange(N, dtype=np.int64)
+    flop = {0: 4 * Hq * D * int((i + 1).sum()), 1: 4 * Hq * D * int(np.minimum(i + 1, S + W).sum())}
+    ms = {}
+    for layer, reps in ((1, 3), (0, 2)):
+        plan.flux_attn_prefill(layer, 0, q, k, v, 0, out)        # warm-up (an SA layer first: 8 ms)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            plan.flux_attn_prefill(layer, 0, q, k, v, 0, out)
+        e1.record()
+        torch.cuda.synchronize()
+        ms[layer] = e0.elapsed_time(e1) / reps
+    assert plan.flux_plan_status() == 0
+    plan.close()
+    del q, k, v, out
+    torch.cuda.empty_cache()
+    tf_fa, tf_sa = flop[0] / ms[0] / 1e9, flop[1] / ms[1] / 1e9
+    n_fa, n_sa = int((synth.layer_masks(w) == 1).sum()), int((synth.layer_masks(w) == 0).sum())
+    return {"workload": "cfg4 prefill: 28/4 heads, d128, batch 1, 131072 tokens in one call per layer, sink 128 + window 4096",
+            "ms_fa_layer": ms[0], "ms_sa_layer": ms[1], "tflops_fa": tf_fa, "tflops_sa": tf_sa,
+            "ms_whole_stack_from_layer_times": n_fa * ms[0] + n_sa * ms[1], "layers": "%d FA + %d SA" % (n_fa, n_sa),
+            "roofline": {"bound": "tensor", "achieved": tf_fa, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                         "frac": tf_fa / peaks["bf16_tflops_sustained"], "frac_of_burst_peak": tf_fa / peaks["bf16_tflops"],
+                         "peak_source": peaks["source"] + " (sustained cuBLAS bf16)", "kernel": "FA prefill layer (0.1 s per launch)",
+                         "traffic": None}}
 
 
 # ---- the paper's two ratios, re-measured on this GPU (context, not the headline) -----------------
@@ -643,6 +750,10 @@ def main():
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-paper-ratios", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true",
+                    help="skip the other decode workloads (cfg4, cfg5) and the 128K prefill layers")
+    ap.add_argument("--sustain-seconds", type=float, default=3.0,
+                    help="after the K timed steps, keep replaying the step for this long and report the sustained rate")
     ap.add_argument("--profile", default=None, choices=["decode", "prefill", "heads"],
                     help="run a small case of one kernel with few launches (for ncu captures) and exit")
     args = ap.parse_args()
@@ -677,7 +788,14 @@ def main():
     W_, K_ = max(3, args.warmup), args.steps
     e2e_steps = 0 if args.no_e2e else min(K_, 10)
     roof_steps = min(K_, 20)
-    total_steps = 1 + 2 * W_ + K_ + roof_steps + (2 + e2e_steps if e2e_steps else 0) + 2
+    # room for the sustained block: no step can be faster than its required bytes at the HBM peak
+    probe = DecodeBench.__new__(DecodeBench)
+    probe.w, probe.mask = w, synth.layer_masks(w)
+    probe.ctx_host = (synth.context_lengths(w)[None, :].astype(np.int32) + 1)
+    floor_ms = DecodeBench.bytes_step(probe, 0) / (peaks["hbm_gbs"] * 1e9) * 1e3
+    sus_chunk = max(10, int(round(100.0 / floor_ms)))                    # about 0.1 s of replays per timed chunk
+    sus_cap = 0 if args.sustain_seconds <= 0 else (int(args.sustain_seconds * 1e3 / floor_ms) // sus_chunk + 1) * sus_chunk
+    total_steps = 1 + 2 * W_ + K_ + sus_cap + roof_steps + (2 + e2e_steps if e2e_steps else 0) + 2
     t_build = time.time()
     db = DecodeBench(flux, w, dev, total_steps)
     db.plan.flux_debug_decode_kernel({"auto": flux.FLUX_DECODE_AUTO, "two_launch": flux.FLUX_DECODE_TWO_LAUNCH,
@@ -717,6 +835,25 @@ def main():
     ms = e0.elapsed_time(e1)
     launches = launches_per_step * K_
     alg_bytes = sum(db.bytes_step(s) for s in range(t_first, t_first + K_))
+    # (1b) sustained: the same replay loop kept up for some seconds (power cap reached, clocks settled)
+    sustained = None
+    if sus_cap:
+        sampler2 = ClockSampler(local)
+        if rank == 0:
+            sampler2.start()
+        sus_ms, sus_steps, sus_bytes, wall0 = 0.0, 0, 0, time.perf_counter()
+        while sus_steps < sus_cap and (time.perf_counter() - wall0) < args.sustain_seconds:
+            sus_ms += timed_replays(db, sus_chunk)
+            sus_bytes += sum(db.bytes_step(s_) for s_ in range(t, t + sus_chunk))
+            t += sus_chunk; sus_steps += sus_chunk
+        clocks2 = sampler2.stop() if rank == 0 else None
+        sus_ms = max_over_ranks(dist, [sus_ms], dev)[0]
+        gbs = sus_bytes / (sus_ms * 1e-3) / 1e9
+        sustained = {"value": whole_job_throughput(world, w.batch, sus_steps, sus_ms), "unit": "tokens/s", "steps": sus_steps,
+                     "seconds": sus_ms / 1e3, "ms_per_step": sus_ms / sus_steps, "step_level_gbs": gbs,
+                     "frac_of_hbm_peak": gbs / peaks["hbm_gbs"], "clocks": clocks2,
+                     "note": "graph replays back to back right after the K timed steps; the short region above runs before "
+                             "the power cap bites, this one mostly under it"}
     # (2) the dominant kernel, event-bracketed launch by launch, on the next steps issued one call at a time
     db.plan.flux_profile_enable(roof_steps * w.n_layers + 8)
     r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -778,7 +915,7 @@ def main():
     tr = traffic_note("decode_kernel")
     roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": ach / peaks["hbm_gbs"], "peak_source": peaks["source"] + " (copy bandwidth)",
-            "kernel": "decode_kernel (mixed FA/SA split-K decode, one launch per layer)",
+            "kernel": decode_kernel_name(flux, args.decode_kernel, w.batch),
             "launches_timed": int(kcnt), "avg_launch_ms": per_launch_ms,
             "algorithmic_bytes_per_launch": per_launch_bytes,
             "traffic": None if tr is None else tr.get("dram_bytes_per_algorithmic_byte") * per_launch_bytes,
@@ -788,7 +925,7 @@ def main():
         "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": K_,
         "warmup": W_, "ms_per_step": ms / K_, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic", "config": workload_config(w, db.mask, db.ctx0),
-        "roofline": roof, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+        "roofline": roof, "sustained": sustained, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
         "stepping": "one CUDA graph per decode step (%d kernel launches of this library), replayed %d times; "
                     "issued call by call the same step takes %.3f ms" % (launches_per_step, K_, eager_ms),
         "omega_msr": float((db.mask == 0).mean()),
@@ -807,6 +944,18 @@ def main():
             line["router_frontend"] = router_frontend_block(flux, dev, peaks, W_)
         except Exception as e:  # report, never hide
             line["router_frontend"] = {"error": repr(e)}
+    if not args.no_secondary and world == 1:
+        for name in ("cfg5", "cfg4"):
+            if name == args.workload:
+                continue
+            try:
+                line["decode_" + name] = secondary_decode_block(flux, dev, peaks, name, 50 if name == "cfg5" else 400, W_, args)
+            except Exception as e:  # report, never hide
+                line["decode_" + name] = {"error": repr(e)}
+        try:
+            line["prefill_cfg4_128k"] = prefill_128k_block(flux, dev, peaks, W_)
+        except Exception as e:  # report, never hide
+            line["prefill_cfg4_128k"] = {"error": repr(e)}
     if not args.no_paper_ratios and world == 1:
         try:
             line["paper_ratios_256k"] = paper_ratio_block(flux, dev, W_)
