@@ -105,6 +105,7 @@ WorkspaceLayout workspace_layout(const flux_config &c)
     w.host_v = off;       off = align_up(off + B * c.n_kv_heads * kRowBytes, A);
     w.host_o = off;       off = align_up(off + B * c.n_q_heads * kRowBytes, A);
     w.router = off;       off = align_up(off + ((size_t)2 * c.n_q_heads * kHeadDim + 3 * kRouterMaxWidth) * sizeof(float), A);
+    w.router_sync = off;  off = align_up(off + 4 * sizeof(uint32_t), A);
     w.tickets = off;      off = align_up(off + (size_t)kDecFusedMaxBatch * c.n_kv_heads * sizeof(uint32_t), A);
     w.total = off;
     return w;
@@ -369,6 +370,7 @@ int flux_plan_create(const flux_config *cfg, flux_plan **plan)
     rc = decode_setup(p);
     if (!rc) rc = decode_fused_setup(p);
     if (!rc) rc = prefill_setup(p);
+    if (!rc) rc = router_setup(p);
     if (rc) {
         delete p;
         return rc;
@@ -714,6 +716,13 @@ int flux_plan_status(flux_plan *plan, uint32_t *status_bits, void *stream)
     if (!rc) rc = check_cuda(cudaMemsetAsync(d, 0, sizeof bits, st), "status clear");
     if (!rc) rc = check_cuda(cudaStreamSynchronize(st), "stream synchronize");
     if (rc) return rc;
+    if (bits & FLUX_STATUS_WAIT_EXPIRED) {   // a kernel left early: its arrival counters are not back at zero
+        rc = check_cuda(cudaMemsetAsync((char *)plan->ws + plan->lay.router_sync, 0, 4 * sizeof(uint32_t), st), "counter clear");
+        if (!rc) rc = check_cuda(cudaMemsetAsync((char *)plan->ws + plan->lay.tickets, 0,
+                                                 (size_t)kDecFusedMaxBatch * plan->cfg.n_kv_heads * sizeof(uint32_t), st), "counter clear");
+        if (!rc) rc = check_cuda(cudaStreamSynchronize(st), "stream synchronize");
+        if (rc) return rc;
+    }
     if (status_bits) *status_bits = bits;
     if (bits & FLUX_STATUS_WAIT_EXPIRED)
         return fail(FLUX_E_DEVICE_TIMEOUT, "a device-side wait expired (status 0x%x)", bits);

@@ -39,6 +39,7 @@ struct WorkspaceLayout {
     size_t host_v;       // bf16  [max_batch][Hkv][D]
     size_t host_o;       // bf16  [max_batch][Hq][D]
     size_t router;       // fp32  [2*Hq*D + 3*kRouterMaxWidth] pooled descriptor and hidden activations
+    size_t router_sync;  // uint32 [4] barrier counters and ticket of the one-launch router front end (zero between launches)
     size_t tickets;      // uint32 [kDecFusedMaxBatch][Hkv] arrival counters of the single-launch decode (zero between launches)
     size_t total;
     int64_t slots;
@@ -122,5 +123,6 @@ int launch_wait_probe(flux_plan *p, long long limit_cycles, cudaStream_t st);
 int decode_setup(flux_plan *p);   // one-time attribute setting for the decode kernels
 int decode_fused_setup(flux_plan *p);
 int prefill_setup(flux_plan *p);
+int router_setup(flux_plan *p);
 
 }  // namespace flux
