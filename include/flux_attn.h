@@ -306,16 +306,6 @@ int flux_profile_enable(flux_plan *plan, int32_t max_records);
 int flux_profile_read(flux_plan *plan, int32_t kind, double *total_ms, int64_t *launches,
                       void *stream);
 
-/* Which kernel flux_attn_prefill launches.  FLUX_PREFILL_AUTO (the default) and
- * FLUX_PREFILL_TCGEN05 run the tcgen05 / TMEM / TMA kernel; FLUX_PREFILL_WARP_MMA runs
- * the warp-level mma.sync kernel (kept for comparison).  Both compute Eq. 1 / Eq. 2 and
- * serve every shape. */
-#define FLUX_PREFILL_AUTO     0
-#define FLUX_PREFILL_WARP_MMA 1
-#define FLUX_PREFILL_TCGEN05  2
-#define FLUX_PREFILL_TCGEN05_PAIR 3  /* CTA pairs sharing K / V tiles; group sizes that are multiples of 4, else as 2 */
-int flux_debug_prefill_kernel(flux_plan *plan, int32_t which);
-
 /* Launch overlap for the single-launch decode kernel (off by default).  With it on, a decode launch
  * builds its schedule and requests its first K / V tiles while the previous kernel in the stream is
  * still draining, and waits for that kernel only before it reads the query rows, the newest K / V row

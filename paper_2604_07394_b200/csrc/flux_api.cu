@@ -529,16 +529,6 @@ int flux_debug_wait_probe(flux_plan *plan, int64_t limit_cycles, void *stream)
     return launch_wait_probe(plan, limit_cycles, (cudaStream_t)stream);
 }
 
-int flux_debug_prefill_kernel(flux_plan *plan, int32_t which)
-{
-    int rc = need_plan(plan, false);
-    if (rc) return rc;
-    if (which < FLUX_PREFILL_AUTO || which > FLUX_PREFILL_TCGEN05_PAIR)
-        return fail(FLUX_E_INVALID_ARG, "unknown prefill kernel selector %d", which);
-    plan->prefill_kernel = which;
-    return FLUX_OK;
-}
-
 int flux_plan_set_launch_overlap(flux_plan *plan, int32_t on)
 {
     int rc = need_plan(plan, false);

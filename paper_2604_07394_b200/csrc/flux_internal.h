@@ -80,7 +80,6 @@ struct flux_plan {
     uint32_t *touch;        // optional device bitmap of the KV rows read (flux_debug_touched), NULL = off
     int32_t touch_words;    // 32-bit words per request
     int dec_ctas;
-    int prefill_kernel;     // FLUX_PREFILL_*
     int decode_kernel;      // FLUX_DECODE_*
     int launch_overlap;     // flux_plan_set_launch_overlap
     // optional per-kernel timing (host-side event pool)

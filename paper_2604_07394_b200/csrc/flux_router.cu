@@ -14,6 +14,7 @@
 // the kernel's shared memory take five separate launches instead.
 #include "flux_internal.h"
 #include "flux_mma_util.h"
+#include "flux_tc_util.h"
 
 namespace flux {
 namespace {
@@ -160,7 +161,8 @@ __device__ __forceinline__ void linear_stage(const __nv_bfloat16 *__restrict__ W
     for (int row = row0; row < n_out; row += warps) {
         const bool staged = pre != nullptr && row == row0;
         const uint4 *w = staged ? reinterpret_cast<const uint4 *>(pre) : reinterpret_cast<const uint4 *>(W + (size_t)row * n_in);
-        float acc = 0.f;
+        // four independent partial sums per lane (one per pair of weights of a 16-byte piece), added in a fixed order
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll 4
         for (int i = lane; i < n_in / 8; i += 32) {
             const uint4 p = staged ? w[i] : __ldg(w + i);
@@ -169,15 +171,12 @@ __device__ __forceinline__ void linear_stage(const __nv_bfloat16 *__restrict__ W
             const float2 w1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&p.y));
             const float2 w2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&p.z));
             const float2 w3 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&p.w));
-            acc = fmaf(w0.x, x0.x, acc);
-            acc = fmaf(w0.y, x0.y, acc);
-            acc = fmaf(w1.x, x0.z, acc);
-            acc = fmaf(w1.y, x0.w, acc);
-            acc = fmaf(w2.x, x1.x, acc);
-            acc = fmaf(w2.y, x1.y, acc);
-            acc = fmaf(w3.x, x1.z, acc);
-            acc = fmaf(w3.y, x1.w, acc);
+            a0 = fmaf(w0.y, x0.y, fmaf(w0.x, x0.x, a0));
+            a1 = fmaf(w1.y, x0.w, fmaf(w1.x, x0.z, a1));
+            a2 = fmaf(w2.y, x1.y, fmaf(w2.x, x1.x, a2));
+            a3 = fmaf(w3.y, x1.w, fmaf(w3.x, x1.z, a3));
         }
+        float acc = (a0 + a1) + (a2 + a3);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
         if (lane == 0) {
@@ -193,24 +192,35 @@ __global__ void __launch_bounds__(256) router_fused_kernel(RouterArgs a)
     __shared__ float2 part[8][32];
     __shared__ int s_abort;
     __shared__ unsigned s_ticket;
+    __shared__ __align__(8) unsigned long long s_bar[3];   // weight rows of stage 1 / 2 / 3 have landed
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) s_abort = 0;
     // ---- the weights do not depend on anything computed here: every warp requests the first row it will need in
     //      each stage right away (one group of asynchronous copies per stage), so the 21 MB are in flight while the
     //      pooling and the first barrier run ----
     unsigned char *pre = reinterpret_cast<unsigned char *>(xs + a.xs_floats) + (size_t)warp * a.pre_bytes;
-    {
+    const uint32_t bar0 = smem_u32(s_bar);
+    if (tid == 0) {
+        for (int s = 0; s < 3; ++s) tc::mbar_init(bar0 + 8 * s, 8);           // one arrival per warp
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    if (lane == 0) {
         const int row0 = (int)((blockIdx.x * blockDim.x + tid) >> 5);
         const __nv_bfloat16 *Ws[3] = {a.w1, a.w2, a.w3};
         const int n_in[3] = {a.F, a.E, a.E}, n_out[3] = {a.E, a.E, a.R};
 #pragma unroll
         for (int s = 0; s < 3; ++s) {
-            if (a.pre_off[s] >= 0 && row0 < n_out[s]) {
-                const unsigned char *src = reinterpret_cast<const unsigned char *>(Ws[s] + (size_t)row0 * n_in[s]);
-                const uint32_t dst = smem_u32(pre + a.pre_off[s]);
-                for (int i = lane; i < n_in[s] / 8; i += 32) cp_async16(dst + i * 16, src + (size_t)i * 16, 16);
+            if (a.pre_off[s] >= 0 && row0 < n_out[s]) {       // one bulk copy per row: n_in * 2 bytes, 16-byte aligned
+                const uint32_t bytes = (uint32_t)n_in[s] * 2u;
+                tc::mbar_expect_tx(bar0 + 8 * s, bytes);
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];\n"
+                             ::"r"(smem_u32(pre + a.pre_off[s])), "l"(Ws[s] + (size_t)row0 * n_in[s]), "r"(bytes), "r"(bar0 + 8 * s)
+                             : "memory");
+            } else {
+                tc::mbar_arrive(bar0 + 8 * s);
             }
-            cp_async_commit();
         }
     }
     // ---- pooling: a CTA takes 32 bf16x2 columns of one segment at a time; warp w sums tokens w, w + 8, ... ----
@@ -242,18 +252,26 @@ __global__ void __launch_bounds__(256) router_fused_kernel(RouterArgs a)
             reinterpret_cast<float2 *>(a.f)[(size_t)seg * a.F2 + col] = make_float2(sum.x * inv, sum.y * inv);
         }
     }
-    // (a CTA that leaves early at a barrier still has copies in flight: they are waited for first)
-    if (!grid_barrier(a.sync + 0, a.status, &s_abort)) { cp_async_wait<0>(); return; }
-    cp_async_wait<2>();
-    __syncwarp();
+    // A CTA that gives up at a barrier still has copies in flight into its shared memory: it waits for them first
+    // (bounded: the weights' arrival does not depend on any other CTA).
+    auto rows_landed = [&](int s) -> bool {
+        bool ok = tc::mbar_try(bar0 + 8 * s, 0u);
+        for (const long long t0 = clock64(); !ok && clock64() - t0 < kRouterWaitCycles;) ok = tc::mbar_try(bar0 + 8 * s, 0u);
+        if (!ok) {
+            atomicOr(a.status, FLUX_STATUS_WAIT_EXPIRED);
+            s_abort = 1;
+        }
+        return __all_sync(0xffffffffu, ok);
+    };
+    auto leave = [&]() { for (int s = 0; s < 3; ++s) rows_landed(s); };
+    if (!grid_barrier(a.sync + 0, a.status, &s_abort)) { leave(); return; }
+    if (!rows_landed(0)) { leave(); return; }
     linear_stage(a.w1, a.b1, a.f, a.h1, a.F, a.E, 1, xs, a.pre_off[0] >= 0 ? pre + a.pre_off[0] : nullptr);
-    if (!grid_barrier(a.sync + 1, a.status, &s_abort)) { cp_async_wait<0>(); return; }
-    cp_async_wait<1>();
-    __syncwarp();
+    if (!grid_barrier(a.sync + 1, a.status, &s_abort)) { leave(); return; }
+    if (!rows_landed(1)) { leave(); return; }
     linear_stage(a.w2, a.b2, a.h1, a.u, a.E, a.E, 0, xs, a.pre_off[1] >= 0 ? pre + a.pre_off[1] : nullptr);
-    if (!grid_barrier(a.sync + 2, a.status, &s_abort)) { cp_async_wait<0>(); return; }
-    cp_async_wait<0>();
-    __syncwarp();
+    if (!grid_barrier(a.sync + 2, a.status, &s_abort)) { leave(); return; }
+    if (!rows_landed(2)) { leave(); return; }
     linear_stage(a.w3, a.b3, a.u, a.h2, a.E, a.R, 1, xs, a.pre_off[2] >= 0 ? pre + a.pre_off[2] : nullptr);
     // ---- the two logits: by the CTA that finishes the stage above last ----
     __syncthreads();

@@ -34,10 +34,6 @@ FLUX_STATUS_WAIT_EXPIRED = 8
 FLUX_KERNEL_DECODE = 0
 FLUX_KERNEL_PREFILL = 1
 
-FLUX_PREFILL_AUTO = 0
-FLUX_PREFILL_WARP_MMA = 1
-FLUX_PREFILL_TCGEN05 = 2
-FLUX_PREFILL_TCGEN05_PAIR = 3
 FLUX_DECODE_AUTO = 0
 FLUX_DECODE_TWO_LAUNCH = 1
 FLUX_DECODE_SINGLE_LAUNCH = 2
@@ -49,7 +45,7 @@ EXPORTS = [
     "flux_plan_create", "flux_plan_destroy", "flux_workspace_size", "flux_plan_set_workspace",
     "flux_router_apply", "flux_router_forward", "flux_attn_prefill", "flux_attn_prefill_blocks", "flux_kv_retain", "flux_kv_append",
     "flux_attn_decode", "flux_attn_decode_heads", "flux_attn_decode_step", "flux_attn_decode_noalloc", "flux_attn_decode_host", "flux_attn_prefill_host", "flux_plan_status",
-    "flux_debug_dispatch", "flux_debug_touched", "flux_debug_prefill_kernel", "flux_debug_decode_kernel", "flux_plan_set_launch_overlap", "flux_debug_wait_probe", "flux_profile_enable", "flux_profile_read", "flux_launch_count", "flux_last_error", "flux_version",
+    "flux_debug_dispatch", "flux_debug_touched", "flux_debug_decode_kernel", "flux_plan_set_launch_overlap", "flux_debug_wait_probe", "flux_profile_enable", "flux_profile_read", "flux_launch_count", "flux_last_error", "flux_version",
 ]
 
 
@@ -111,7 +107,6 @@ def load():
     L.flux_attn_prefill_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, i32, i32, vp, vp, vp]
     L.flux_plan_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32), vp]
     L.flux_debug_dispatch.argtypes = [vp, vp, i32, ctypes.POINTER(i32), vp]
-    L.flux_debug_prefill_kernel.argtypes = [vp, i32]
     L.flux_debug_decode_kernel.argtypes = [vp, i32]
     L.flux_plan_set_launch_overlap.argtypes = [vp, i32]
     L.flux_debug_touched.argtypes = [vp, vp, i32]
@@ -302,9 +297,6 @@ class Plan:
 
     def flux_debug_wait_probe(self, limit_cycles: int) -> None:
         _check(load().flux_debug_wait_probe(self._h, limit_cycles, _stream()))
-
-    def flux_debug_prefill_kernel(self, which: int) -> None:
-        _check(load().flux_debug_prefill_kernel(self._h, which))
 
     def flux_plan_set_launch_overlap(self, on: bool) -> None:
         _check(load().flux_plan_set_launch_overlap(self._h, 1 if on else 0))

@@ -30,7 +30,6 @@ def _random_mask(nb, density, seed):
     return np.tril(bm)
 
 
-@pytest.mark.parametrize("kernel", [2, 1], ids=["tcgen05", "warp_mma"])
 @pytest.mark.parametrize("N,Hq,Hkv,density,chunks", [
     (64, 4, 2, 0.5, None),
     (130, 7, 1, 0.4, None),
@@ -39,10 +38,9 @@ def _random_mask(nb, density, seed):
     (1000, 6, 2, 0.2, (0, 512, 1000)),
     (900, 3, 3, 0.15, (0, 64, 320, 900)),
 ])
-def test_block_mask_prefill_small_shapes(flux, N, Hq, Hkv, density, chunks, kernel):
+def test_block_mask_prefill_small_shapes(flux, N, Hq, Hkv, density, chunks):
     nb = -(-N // B)
     plan = flux.Plan(flux.make_config(1, Hq, Hkv, 0, 1, 1, 1024), DEV)
-    plan.flux_debug_prefill_kernel(kernel)
     q = synth.normal_bf16((N, Hq, 128), 2000 + N, 1, DEV)
     k = synth.normal_bf16((N, Hkv, 128), 2000 + N, 2, DEV)
     v = synth.normal_bf16((N, Hkv, 128), 2000 + N, 3, DEV)
@@ -60,12 +58,10 @@ def test_block_mask_prefill_small_shapes(flux, N, Hq, Hkv, density, chunks, kern
     assert plan.flux_plan_status() == 0
 
 
-@pytest.mark.parametrize("kernel", [2, 1], ids=["tcgen05", "warp_mma"])
-def test_full_block_mask_equals_fa_and_empty_row_is_flagged(flux, kernel):
+def test_full_block_mask_equals_fa_and_empty_row_is_flagged(flux):
     N, Hq, Hkv = 200, 4, 2
     nb = -(-N // B)
     plan = flux.Plan(flux.make_config(1, Hq, Hkv, 0, 1, 1, 1024), DEV)
-    plan.flux_debug_prefill_kernel(kernel)
     plan.flux_router_apply(mask=np.array([[1]], dtype=np.uint8))
     q = synth.normal_bf16((N, Hq, 128), 77, 1, DEV)
     k = synth.normal_bf16((N, Hkv, 128), 77, 2, DEV)
@@ -85,14 +81,12 @@ def test_full_block_mask_equals_fa_and_empty_row_is_flagged(flux, kernel):
         plan.flux_attn_prefill_blocks(q[10:], k, v, 10, torch.from_numpy(tri).to(DEV))
 
 
-@pytest.mark.parametrize("kernel", [2, 1], ids=["tcgen05", "warp_mma"])
-def test_streaming_block_mask_at_32k_sampled_rows(flux, kernel):
+def test_streaming_block_mask_at_32k_sampled_rows(flux):
     """cfg2 shapes (32K tokens, 32/8 heads), sink 128 + window 2048 as 2 + 32 blocks of 64."""
     w = synth.WORKLOADS["cfg2"]
     N, Hq, Hkv, S, W = w.prompt_len, w.n_q_heads, w.n_kv_heads, w.sink, w.window
     nb = N // B
     plan = flux.Plan(flux.make_config(1, Hq, Hkv, S, W, 1, N), DEV)
-    plan.flux_debug_prefill_kernel(kernel)
     q = synth.normal_bf16((N, Hq, 128), w.seed, synth.stream_id("q"), DEV)
     k = synth.normal_bf16((N, Hkv, 128), w.seed, synth.stream_id("k"), DEV)
     v = synth.normal_bf16((N, Hkv, 128), w.seed, synth.stream_id("v"), DEV)

@@ -28,8 +28,8 @@ def _sample_heads(Hq, G):
     return sorted({0, G - 1, G, Hq // 2, Hq - G, Hq - 1} & set(range(Hq)))
 
 
-@pytest.mark.parametrize("cfg,kernel", [("cfg2", 0), ("cfg2", 1), ("cfg2", 3), ("cfg4", 0)])
-def test_prefill_full_size_sampled_rows(flux, cfg, kernel):
+@pytest.mark.parametrize("cfg", ["cfg2", "cfg4"])
+def test_prefill_full_size_sampled_rows(flux, cfg):
     """cfg2: 32K tokens, 32/8 heads, sink 128 + window 2048; cfg4: 128K tokens, 28/4 heads (7 query
     heads per KV head), sink 128 + window 4096.  One FA and one SA layer each, whole prompt in one
     call (as the benchmark does) and, for cfg2, also in chunks of 16384 (Appendix D.3 chunk size)."""
@@ -37,7 +37,6 @@ def test_prefill_full_size_sampled_rows(flux, cfg, kernel):
     N, Hq, Hkv, S, W = w.prompt_len, w.n_q_heads, w.n_kv_heads, w.sink, w.window
     plan = flux.Plan(flux.make_config(2, Hq, Hkv, S, W, 1, N), DEV)
     plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
-    plan.flux_debug_prefill_kernel(kernel)
     q = synth.normal_bf16((N, Hq, 128), w.seed, synth.stream_id("q"), DEV)
     k = synth.normal_bf16((N, Hkv, 128), w.seed, synth.stream_id("k"), DEV)
     v = synth.normal_bf16((N, Hkv, 128), w.seed, synth.stream_id("v"), DEV)
@@ -51,7 +50,7 @@ def test_prefill_full_size_sampled_rows(flux, cfg, kernel):
         out = plan.flux_attn_prefill(layer, 0, q, k, v, 0)
         rec = plan.flux_debug_dispatch(1)
         got = out[torch.from_numpy(rr).to(DEV), torch.from_numpy(hh).to(DEV)]
-        compare(got, ref, "%s prefill mode %d kernel %d" % (cfg, mode, kernel))
+        compare(got, ref, "%s prefill mode %d" % (cfg, mode))
         assert rec[0, 0] == mode and rec[0, 3] == N
         assert expand_ranges(rec[0]) == oracle.kept(mode, N - 1, S, W).tolist()
         if cfg == "cfg2":
@@ -59,7 +58,7 @@ def test_prefill_full_size_sampled_rows(flux, cfg, kernel):
             for a in range(0, N, 16384):
                 out2[a:a + 16384] = plan.flux_attn_prefill(layer, 0, q[a:a + 16384], k[:a + 16384], v[:a + 16384], a)
             got2 = out2[torch.from_numpy(rr).to(DEV), torch.from_numpy(hh).to(DEV)]
-            compare(got2, ref, "%s chunked prefill mode %d kernel %d" % (cfg, mode, kernel))
+            compare(got2, ref, "%s chunked prefill mode %d" % (cfg, mode))
     assert plan.flux_plan_status() == 0
 
 
@@ -134,7 +133,7 @@ def test_decode_full_size_sampled(flux, cfg, dk):
 
 def test_sparse_outputs_ignore_keys_outside_the_kept_set_at_full_size(flux):
     """A property that needs no oracle and holds at any size: changing K and V at positions a query does
-    not keep must leave its output bit-identical.  32K prefill (both tensor-core kernels) and a 64K
+    not keep must leave its output bit-identical.  32K prefill and a 64K
     decode in the full cache layout; the FA layer, which keeps those positions, must change."""
     w = synth.WORKLOADS["cfg2"]
     N, Hq, Hkv, S, W = w.prompt_len, w.n_q_heads, w.n_kv_heads, w.sink, w.window
@@ -148,16 +147,14 @@ def test_sparse_outputs_ignore_keys_outside_the_kept_set_at_full_size(flux):
     k2[a:b] = synth.normal_bf16((b - a, Hkv, 128), 99, 1, DEV)
     v2[a:b] = synth.normal_bf16((b - a, Hkv, 128), 99, 2, DEV)
     first_unaffected = b - 1 + W                        # the first query whose window starts after b - 1
-    for kernel in (2, 3):
-        plan.flux_debug_prefill_kernel(kernel)
-        sa0, sa1 = plan.flux_attn_prefill(1, 0, q, k, v, 0), plan.flux_attn_prefill(1, 0, q, k2, v2, 0)
-        assert torch.equal(sa0[:a].view(torch.int16), sa1[:a].view(torch.int16))
-        assert torch.equal(sa0[first_unaffected:].view(torch.int16), sa1[first_unaffected:].view(torch.int16))
-        assert not torch.equal(sa0[a:first_unaffected].view(torch.int16), sa1[a:first_unaffected].view(torch.int16))
-        fa0, fa1 = plan.flux_attn_prefill(0, 0, q, k, v, 0), plan.flux_attn_prefill(0, 0, q, k2, v2, 0)
-        assert torch.equal(fa0[:a].view(torch.int16), fa1[:a].view(torch.int16))
-        changed = (fa0[b:] != fa1[b:]).flatten(1).any(dim=1)
-        assert bool(changed.all())                      # every later FA row sees the rewritten keys
+    sa0, sa1 = plan.flux_attn_prefill(1, 0, q, k, v, 0), plan.flux_attn_prefill(1, 0, q, k2, v2, 0)
+    assert torch.equal(sa0[:a].view(torch.int16), sa1[:a].view(torch.int16))
+    assert torch.equal(sa0[first_unaffected:].view(torch.int16), sa1[first_unaffected:].view(torch.int16))
+    assert not torch.equal(sa0[a:first_unaffected].view(torch.int16), sa1[a:first_unaffected].view(torch.int16))
+    fa0, fa1 = plan.flux_attn_prefill(0, 0, q, k, v, 0), plan.flux_attn_prefill(0, 0, q, k2, v2, 0)
+    assert torch.equal(fa0[:a].view(torch.int16), fa1[:a].view(torch.int16))
+    changed = (fa0[b:] != fa1[b:]).flatten(1).any(dim=1)
+    assert bool(changed.all())                      # every later FA row sees the rewritten keys
     # decode at 65536 tokens, full layout: rewrite everything between the sink and the window
     n = 65536
     kc = synth.normal_bf16((n, Hkv, 128), 7, 1, DEV)

@@ -141,17 +141,15 @@ PREFILL_CASES = [
     (300, 4, 4, 64, 100, None),           # one query head per KV head: a CTA pairs two row tiles of a head
     (640, 5, 5, 128, 128, (0, 256, 640)),
     (129, 1, 1, 5, 9, None),
-    (1000, 16, 2, 64, 256, (0, 384, 1000)),     # eight query heads per KV head: two head quads for the CTA-pair kernel
+    (1000, 16, 2, 64, 256, (0, 384, 1000)),     # eight query heads per KV head: four head pairs per KV head
     (900, 12, 3, 0, 130, None),
 ]
 
 
-@pytest.mark.parametrize("kernel", [2, 1, 3], ids=["tcgen05", "warp_mma", "tcgen05_pair"])
 @pytest.mark.parametrize("N,Hq,Hkv,S,W,chunks", PREFILL_CASES)
-def test_prefill_small_shapes(flux, N, Hq, Hkv, S, W, chunks, kernel):
+def test_prefill_small_shapes(flux, N, Hq, Hkv, S, W, chunks):
     plan = _plan(flux, 2, Hq, Hkv, S, W, 1, 1024)
     plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
-    plan.flux_debug_prefill_kernel(kernel)
     seed = 1000 + N
     q = synth.normal_bf16((N, Hq, 128), seed, 1, DEV)
     k = synth.normal_bf16((N, Hkv, 128), seed, 2, DEV)
@@ -170,15 +168,13 @@ def test_prefill_small_shapes(flux, N, Hq, Hkv, S, W, chunks, kernel):
     assert plan.flux_plan_status() == 0
 
 
-@pytest.mark.parametrize("kernel", [2, 1, 3], ids=["tcgen05", "warp_mma", "tcgen05_pair"])
-def test_prefill_scores_rising_along_the_sequence(flux, kernel):
+def test_prefill_scores_rising_along_the_sequence(flux):
     """Keys whose scores grow by tens of log2 units from one KV tile to the next, so the running
     maximum has to be raised (and the accumulator rescaled) again and again in the middle of a row;
     and the mirror case, where the first keys dominate and later tiles underflow to nothing."""
     N, Hq, Hkv, S, W = 1100, 8, 2, 64, 300
     plan = _plan(flux, 2, Hq, Hkv, S, W, 1, 2048)
     plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
-    plan.flux_debug_prefill_kernel(kernel)
     q = synth.normal_bf16((N, Hq, 128), 4242, 1, DEV).float() + 1.0
     v = synth.normal_bf16((N, Hkv, 128), 4242, 3, DEV)
     ramp = torch.linspace(0.0, 3.0, N, device=DEV)[:, None, None]
