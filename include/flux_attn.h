@@ -306,6 +306,30 @@ int flux_profile_enable(flux_plan *plan, int32_t max_records);
 int flux_profile_read(flux_plan *plan, int32_t kind, double *total_ms, int64_t *launches,
                       void *stream);
 
+/* A decode step evaluated in pieces over disjoint key ranges, and the merge of the pieces: the building blocks for
+ * spreading one long context over several GPUs (each holds a range of the cache rows, evaluates its piece, the
+ * pieces are exchanged -- B * n_q_heads * 130 floats per piece -- and merged).  Eq. 1 / Eq. 2 are sums over keys,
+ * so pieces over disjoint key sets merge exactly, by rescaling with the difference of their maxima.
+ *
+ * flux_attn_decode_partial: as flux_attn_decode, restricted per request to the key positions
+ * [key_begin[b], key_end[b]) (device int32 arrays; clamped to [0, ctx_len[b]]).  A request that reads its rows
+ * densely (FA, or SA while sink + window still cover the context) reads exactly those rows; a sparse request is
+ * evaluated whole by the call whose range holds its newest position ctx_len[b] - 1 and yields an empty piece in
+ * every other call.  Instead of an output row the call writes, for every (request, query head), the piece
+ *   part_o  fp32 [B][n_q_heads][head_dim]  sum over the range's kept keys of 2^(s_j - m) V_j   (not normalised)
+ *   part_ml fp32 [B][n_q_heads][2]         m = the maximum scaled score in log2 units (s_j = scale * log2(e) * q.k_j;
+ *                                          -1e30 for an empty piece), l = sum of 2^(s_j - m)
+ * both device memory.  Always runs the two-launch kernels.
+ *
+ * flux_attn_combine: merges n_sets pieces laid out [n_sets][B][n_q_heads][...] (what an all-gather of the ranks'
+ * pieces produces) into out bf16 [B][n_q_heads][head_dim]: m = max m_s, O = sum_s O_s 2^(m_s - m), l likewise,
+ * out = O / l (a row whose pieces are all empty is zero). */
+int flux_attn_decode_partial(flux_plan *plan, int32_t layer, int32_t B, const void *q, const void *const *k_caches,
+                             const void *const *v_caches, const int32_t *ctx_len, const int32_t *key_begin,
+                             const int32_t *key_end, float *part_o, float *part_ml, void *stream);
+int flux_attn_combine(flux_plan *plan, int32_t B, int32_t n_sets, const float *part_o, const float *part_ml, void *out,
+                      void *stream);
+
 /* Launch overlap for the single-launch decode kernel (off by default).  With it on, a decode launch
  * builds its schedule and requests its first K / V tiles while the previous kernel in the stream is
  * still draining, and waits for that kernel only before it reads the query rows, the newest K / V row

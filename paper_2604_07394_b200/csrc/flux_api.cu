@@ -603,6 +603,36 @@ int flux_attn_decode(flux_plan *plan, int32_t layer, int32_t B, const void *q,
     return launch_decode(plan, layer, B, q, k_caches, v_caches, ctx_len, out, (cudaStream_t)stream);
 }
 
+int flux_attn_decode_partial(flux_plan *plan, int32_t layer, int32_t B, const void *q, const void *const *k_caches,
+                             const void *const *v_caches, const int32_t *ctx_len, const int32_t *key_begin,
+                             const int32_t *key_end, float *part_o, float *part_ml, void *stream)
+{
+    int rc = check_batch_call(plan, layer, B);
+    if (rc) return rc;
+    if (!q || !k_caches || !v_caches || !ctx_len || !key_begin || !key_end || !part_o || !part_ml)
+        return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    if (!aligned16(q) || !aligned16(part_o) || (((uintptr_t)part_ml) & 7u))
+        return fail(FLUX_E_INVALID_ARG, "q / part_o must be 16-byte aligned, part_ml 8-byte aligned");
+    if (!is_device_ptr(key_begin) || !is_device_ptr(key_end) || !is_device_ptr(part_o) || !is_device_ptr(part_ml))
+        return fail(FLUX_E_INVALID_ARG, "key ranges and partial outputs must be device memory");
+    const DecPartial part = {key_begin, key_end, part_o, part_ml};
+    return launch_decode(plan, layer, B, q, k_caches, v_caches, ctx_len, nullptr, (cudaStream_t)stream, nullptr, nullptr,
+                         nullptr, &part);
+}
+
+int flux_attn_combine(flux_plan *plan, int32_t B, int32_t n_sets, const float *part_o, const float *part_ml, void *out,
+                      void *stream)
+{
+    int rc = need_plan(plan, false);
+    if (rc) return rc;
+    if (B < 1 || B > plan->cfg.max_batch) return fail(FLUX_E_CAPACITY, "B=%d outside [1, %d]", B, plan->cfg.max_batch);
+    if (n_sets < 1 || n_sets > 1024) return fail(FLUX_E_INVALID_ARG, "n_sets=%d outside [1, 1024]", n_sets);
+    if (!part_o || !part_ml || !out) return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    if (!aligned16(part_o) || !aligned16(out) || (((uintptr_t)part_ml) & 7u))
+        return fail(FLUX_E_INVALID_ARG, "part_o / out must be 16-byte aligned, part_ml 8-byte aligned");
+    return launch_combine_sets(plan, part_o, part_ml, n_sets, B * plan->cfg.n_q_heads, out, (cudaStream_t)stream);
+}
+
 int flux_attn_decode_heads(flux_plan *plan, int32_t B, const void *q, const void *const *k_caches,
                            const void *const *v_caches, const int32_t *ctx_len, const uint8_t *head_mask,
                            void *out, void *stream)

@@ -66,6 +66,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
             mode_raw = a.mask[b * a.L + a.layer];
         }
         ReqInfo r = req_info(a.ctx_len[b], mode_raw, a.S, a.W, a.layout, a.max_context, a.status);
+        if (a.key_begin != nullptr) dec_restrict(r, a.key_begin[b], a.key_end[b], a.S, a.W);
         s_neff[b] = r.n_eff;
         s_split[b] = r.split;
         s_shift[b] = r.shift;
@@ -315,8 +316,13 @@ __global__ void __launch_bounds__(kCombWarps * 32) decode_combine_kernel(DecArgs
 
     const int ustart = a.sched[b], uend = a.sched[b + 1], span = a.sched[a.B + 1];
     const int units = uend - ustart;
-    if (units == 0) {  // inactive request
-        if (threadIdx.x < kHeadDim) dst[threadIdx.x] = __float2bfloat16(0.f);
+    float *pdst_o = a.pout_o ? a.pout_o + ((size_t)b * a.Hq + h) * kHeadDim : nullptr;
+    if (units == 0) {  // inactive request (or, in a partial call, no key of the range is kept): nothing to add
+        if (threadIdx.x < kHeadDim) {
+            if (pdst_o) pdst_o[threadIdx.x] = 0.f; else dst[threadIdx.x] = __float2bfloat16(0.f);
+        }
+        if (pdst_o && threadIdx.x == 0)
+            *reinterpret_cast<float2 *>(a.pout_ml + ((size_t)b * a.Hq + h) * 2) = make_float2(kNegBig, 0.f);
         return;
     }
     const int tiles = units / n_hg;
@@ -392,7 +398,41 @@ __global__ void __launch_bounds__(kCombWarps * 32) decode_combine_kernel(DecArgs
         num += s_o[w][d] * sc;
         den += s_l[w] * sc;
     }
-    dst[d] = __float2bfloat16(den > 0.f ? num / den : 0.f);
+    if (pdst_o) {   // partial call: the merged state itself (O unnormalised), for flux_attn_combine
+        pdst_o[d] = num;
+        if (d == 0) *reinterpret_cast<float2 *>(a.pout_ml + ((size_t)b * a.Hq + h) * 2) = make_float2(mm, den);
+    } else {
+        dst[d] = __float2bfloat16(den > 0.f ? num / den : 0.f);
+    }
+}
+
+// Merges n_sets partial evaluations of the same (request, query head) rows -- each (O unnormalised, m, l) over a
+// disjoint set of keys -- into the bf16 output: m = max m_s, O = sum O_s 2^(m_s - m), l likewise, out = O / l.
+// Sets are laid out [set][row]; one warp per row, four channels per lane, the sets taken in order.
+__global__ void __launch_bounds__(256) combine_sets_kernel(const float *__restrict__ po, const float *__restrict__ pml,
+                                                           int n_sets, int n_rows, __nv_bfloat16 *__restrict__ out)
+{
+    const int row = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
+    if (row >= n_rows) return;
+    float m = kNegBig;
+    for (int s = 0; s < n_sets; ++s) m = fmaxf(m, pml[((size_t)s * n_rows + row) * 2]);
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    float l = 0.f;
+    for (int s = 0; s < n_sets; ++s) {
+        const float2 ml = *reinterpret_cast<const float2 *>(pml + ((size_t)s * n_rows + row) * 2);
+        const float w = fast_exp2(ml.x - m);
+        const float4 v = *reinterpret_cast<const float4 *>(po + ((size_t)s * n_rows + row) * kHeadDim + lane * 4);
+        acc.x += v.x * w;
+        acc.y += v.y * w;
+        acc.z += v.z * w;
+        acc.w += v.w * w;
+        l += ml.y * w;
+    }
+    const float inv = l > 0.f ? 1.0f / l : 0.f;
+    uint2 pk;
+    pk.x = pack_bf16(acc.x * inv, acc.y * inv);
+    pk.y = pack_bf16(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2 *>(out + (size_t)row * kHeadDim + lane * 4) = pk;
 }
 
 constexpr int kDecSmemBytes = kDecWarps * kDecStages * kDecStageBytes;
@@ -409,9 +449,16 @@ int decode_setup(flux_plan *p)
                       "cudaFuncSetAttribute(decode_kernel)");
 }
 
+int launch_combine_sets(flux_plan *p, const float *po, const float *pml, int n_sets, int n_rows, void *out, cudaStream_t st)
+{
+    combine_sets_kernel<<<(n_rows + 7) / 8, 256, 0, st>>>(po, pml, n_sets, n_rows, (__nv_bfloat16 *)out);
+    p->launches++;
+    return check_cuda(cudaGetLastError(), "partial-set combine kernel launch");
+}
+
 int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *const *k_caches,
                   const void *const *v_caches, const int32_t *ctx_len, void *out, cudaStream_t st,
-                  const void *k_new, const void *v_new, const uint8_t *head_mask)
+                  const void *k_new, const void *v_new, const uint8_t *head_mask, const DecPartial *part)
 {
     const flux_config &c = p->cfg;
     char *ws = (char *)p->ws;
@@ -437,9 +484,13 @@ int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *con
     a.head_mask = head_mask;
     a.tickets = (uint32_t *)(ws + p->lay.tickets);
     a.overlap = (p->launch_overlap && p->touch == nullptr) ? 1 : 0;   // the debug bitmap is written by the loaders
+    a.key_begin = part ? part->key_begin : nullptr;
+    a.key_end = part ? part->key_end : nullptr;
+    a.pout_o = part ? part->out_o : nullptr;
+    a.pout_ml = part ? part->out_ml : nullptr;
     const int fused_max = p->decode_kernel == FLUX_DECODE_SINGLE_LAUNCH ? kDecFusedMaxBatch
                           : p->decode_kernel == FLUX_DECODE_AUTO        ? kDecFusedAutoBatch : 0;
-    if (head_mask == nullptr && B <= fused_max && c.n_kv_heads <= kDecFusedMaxKvHeads)
+    if (head_mask == nullptr && part == nullptr && B <= fused_max && c.n_kv_heads <= kDecFusedMaxKvHeads)
         return launch_decode_fused(p, a, st);
     const int rec = prof_begin(p, FLUX_KERNEL_DECODE, st);
     decode_kernel<<<p->dec_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
@@ -593,6 +644,8 @@ extern "C" int flux_attn_decode_noalloc(const flux_config *cfg, int32_t layer, i
     a.head_mask = nullptr;
     a.tickets = nullptr;
     a.overlap = 0;
+    a.key_begin = a.key_end = nullptr;
+    a.pout_o = a.pout_ml = nullptr;
     decode_kernel<<<nd->n_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
     rc = check_cuda(cudaGetLastError(), "decode kernel launch");
     if (rc) return rc;

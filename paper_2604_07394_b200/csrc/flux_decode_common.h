@@ -37,6 +37,10 @@ struct DecArgs {
     uint32_t *tickets;
     // single-launch kernel only: schedule and first tile loads before the grid-dependency wait
     int overlap;
+    // partial evaluation over a key range (flux_attn_decode_partial): positions [key_begin[b], key_end[b]) of each
+    // request, and where the merged (O, m, l) of every (request, query head) goes instead of the bf16 output
+    const int32_t *key_begin, *key_end;
+    float *pout_o, *pout_ml;
 };
 
 // What one request contributes to this layer's launch.
@@ -73,6 +77,22 @@ __device__ __forceinline__ ReqInfo req_info(int n_raw, int mode_raw, int S, int 
         }  // COMPACT_SA: the S + W slots are exactly the kept rows, in slot order
     }
     return r;
+}
+
+// Restricts a request to the key positions [kb, ke).  A request that walks its rows densely (FA, or SA while sink +
+// window still cover the context) reads rows kb .. ke - 1; a sparse request is taken whole by the range that holds
+// its newest position and skipped by every other range (its kept rows are few: splitting them gains nothing).
+__device__ __forceinline__ void dec_restrict(ReqInfo &r, int kb, int ke, int S, int W)
+{
+    kb = kb < 0 ? 0 : kb;
+    ke = ke > r.n ? r.n : ke;
+    if (r.mode == 1 || r.n <= S + W) {
+        r.split = 0;
+        r.shift = kb;
+        r.n_eff = ke > kb ? ke - kb : 0;
+    } else if (!(kb <= r.n - 1 && r.n - 1 < ke)) {
+        r.n_eff = 0;
+    }
 }
 
 // Cache row of the token a fused-append launch stores for a request (-1: nothing to store).

@@ -107,10 +107,17 @@ int launch_kv_retain(flux_plan *p, int layer, int req, const void *k_src, const 
                      int n, void *k_cache, void *v_cache, cudaStream_t st);
 // k_new / v_new non-NULL: the launch also appends the newest token (flux_attn_decode_step);
 // head_mask non-NULL: per-KV-head modes [B][Hkv] instead of the routed layer mask (flux_attn_decode_heads)
+// part non-NULL: evaluate only the keys [key_begin[b], key_end[b]) and write the merged (O, m, l) of every
+// (request, query head) to out_o / out_ml instead of the bf16 output (flux_attn_decode_partial)
+struct DecPartial {
+    const int32_t *key_begin, *key_end;
+    float *out_o, *out_ml;
+};
 int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *const *k_caches,
                   const void *const *v_caches, const int32_t *ctx_len, void *out,
                   cudaStream_t st, const void *k_new = nullptr, const void *v_new = nullptr,
-                  const uint8_t *head_mask = nullptr);
+                  const uint8_t *head_mask = nullptr, const DecPartial *part = nullptr);
+int launch_combine_sets(flux_plan *p, const float *po, const float *pml, int n_sets, int n_rows, void *out, cudaStream_t st);
 int launch_prefill(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v,
                    int q_start, int Nq, void *out, cudaStream_t st);
 // bracket a dominant-kernel launch with events when profiling is on

@@ -44,7 +44,7 @@ FLUX_KV_COMPACT_SA = 1
 EXPORTS = [
     "flux_plan_create", "flux_plan_destroy", "flux_workspace_size", "flux_plan_set_workspace",
     "flux_router_apply", "flux_router_forward", "flux_attn_prefill", "flux_attn_prefill_blocks", "flux_kv_retain", "flux_kv_append",
-    "flux_attn_decode", "flux_attn_decode_heads", "flux_attn_decode_step", "flux_attn_decode_noalloc", "flux_attn_decode_host", "flux_attn_prefill_host", "flux_plan_status",
+    "flux_attn_decode", "flux_attn_decode_heads", "flux_attn_decode_partial", "flux_attn_combine", "flux_attn_decode_step", "flux_attn_decode_noalloc", "flux_attn_decode_host", "flux_attn_prefill_host", "flux_plan_status",
     "flux_debug_dispatch", "flux_debug_touched", "flux_debug_decode_kernel", "flux_plan_set_launch_overlap", "flux_debug_wait_probe", "flux_profile_enable", "flux_profile_read", "flux_launch_count", "flux_last_error", "flux_version",
 ]
 
@@ -100,6 +100,8 @@ def load():
     L.flux_kv_retain.argtypes = [vp, i32, i32, vp, vp, i32, vp, vp, vp]
     L.flux_kv_append.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
+    L.flux_attn_decode_partial.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.flux_attn_combine.argtypes = [vp, i32, i32, vp, vp, vp, vp]
     L.flux_attn_decode_heads.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode_noalloc.argtypes = [cfgp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -249,6 +251,25 @@ class Plan:
             out = torch.empty_like(q)
         _check(load().flux_attn_decode(self._h, layer, B, _ptr(q), _ptr(k_caches), _ptr(v_caches),
                                        _ptr(ctx_len), _ptr(out), _stream()))
+        return out
+
+    def flux_attn_decode_partial(self, layer, B, q, k_caches, v_caches, ctx_len, key_begin, key_end, part_o=None, part_ml=None):
+        """One piece of a decode step over the key positions [key_begin[b], key_end[b]) -> (part_o fp32 [B][Hq][D],
+        part_ml fp32 [B][Hq][2])."""
+        if part_o is None:
+            part_o = torch.empty((B, self.cfg.n_q_heads, 128), dtype=torch.float32, device=self.device)
+        if part_ml is None:
+            part_ml = torch.empty((B, self.cfg.n_q_heads, 2), dtype=torch.float32, device=self.device)
+        _check(load().flux_attn_decode_partial(self._h, layer, B, _ptr(q), _ptr(k_caches), _ptr(v_caches), _ptr(ctx_len),
+                                               _ptr(key_begin), _ptr(key_end), _ptr(part_o), _ptr(part_ml), _stream()))
+        return part_o, part_ml
+
+    def flux_attn_combine(self, B, part_o, part_ml, out=None):
+        """part_o fp32 [n_sets][B][Hq][D], part_ml fp32 [n_sets][B][Hq][2] -> out bf16 [B][Hq][D]."""
+        n_sets = int(part_o.shape[0])
+        if out is None:
+            out = torch.empty((B, self.cfg.n_q_heads, 128), dtype=torch.bfloat16, device=self.device)
+        _check(load().flux_attn_combine(self._h, B, n_sets, _ptr(part_o), _ptr(part_ml), _ptr(out), _stream()))
         return out
 
     def flux_attn_decode_heads(self, B, q, k_caches, v_caches, ctx_len, head_mask, out=None):
