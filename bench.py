@@ -295,7 +295,7 @@ def kernel_roofline(db, flux, t, steps, peaks, kernel_name):
 
 
 def decode_kernel_name(flux, plan_choice, batch):
-    single = plan_choice == "single_launch" and batch <= 8 or plan_choice == "auto" and batch <= 4
+    single = plan_choice != "two_launch" and batch <= 32
     return ("decode_fused_kernel (split-K decode and merge in one launch per layer)" if single else
             "decode_kernel (mixed FA/SA split-K decode, one launch per layer)")
 
@@ -542,6 +542,7 @@ def paper_ratio_block(flux, dev, warmup):
     for name, w in (("dense", dataclasses.replace(base, mask_rule="fixed", mask_arg=tuple([1] * L))),
                     ("routed", base)):
         db = DecodeBench(flux, w, dev, steps + warmup + 4, host_mirrors=False)
+        db.plan.flux_plan_set_launch_overlap(True)
         t = 0
         db.step(t); t += 1
         db.capture_step(t)
@@ -607,6 +608,7 @@ def head_level_block(flux, dev, peaks, warmup, n=262144, reps=30):
     w = synth.WORKLOADS["cfg3"]
     Hq, Hkv, S, W = w.n_q_heads, w.n_kv_heads, 128, 2048
     plan = flux.Plan(flux.make_config(2, Hq, Hkv, S, W, 1, n), dev)
+    plan.flux_debug_decode_kernel(flux.FLUX_DECODE_TWO_LAUNCH)     # the kernels the head-level mode runs: like against like
     plan.flux_router_apply(mask=np.array([[1, 0]], dtype=np.uint8))
     # two cache sets, used alternately, so that no call finds its rows in L2 (a sparse layer's 17 MB would fit)
     sets = []
@@ -734,6 +736,33 @@ def profile_case(flux, dev, which):
         assert db.plan.flux_plan_status() == 0
         print(json.dumps({"profile_case": "decode", "layers": 2, "launch_bytes": db.bytes_step(0) / 2,
                           "cache_gb": db.cache_bytes / 1e9}))
+    elif which == "decode_b1":  # batch 1, 28/4 heads, 128K context: one dense and one sparse layer, a few steps
+        w = dataclasses.replace(synth.WORKLOADS["cfg4"], n_layers=2, prompt_len=0, mask_rule="fixed", mask_arg=(1, 0))
+        db = DecodeBench(flux, w, dev, 6, host_mirrors=False)
+        db.plan.flux_plan_set_launch_overlap(True)
+        for t in range(4):
+            db.step(t)
+        torch.cuda.synchronize()
+        assert db.plan.flux_plan_status() == 0
+        print(json.dumps({"profile_case": "decode_b1", "launch_order": "dense, sparse, repeated 4 times",
+                          "dense_launch_bytes": int(db.kept_rows(0)[0, 0]) * 2 * w.n_kv_heads * D * 2,
+                          "sparse_launch_bytes": int(db.kept_rows(0)[0, 1]) * 2 * w.n_kv_heads * D * 2}))
+    elif which == "prefill32k":  # the benchmark's own FA layer: 32768 tokens, one warm-up launch and one more
+        w = synth.WORKLOADS["cfg2"]
+        N = w.prompt_len
+        plan = flux.Plan(flux.make_config(1, w.n_q_heads, w.n_kv_heads, w.sink, w.window, 1, N), dev)
+        plan.flux_router_apply(mask=np.array([[1]], dtype=np.uint8))
+        q = synth.normal_bf16((N, w.n_q_heads, D), w.seed, synth.stream_id("q"), dev)
+        k = synth.normal_bf16((N, w.n_kv_heads, D), w.seed, synth.stream_id("k"), dev)
+        v = synth.normal_bf16((N, w.n_kv_heads, D), w.seed, synth.stream_id("v"), dev)
+        out = torch.empty_like(q)
+        for _ in range(2):
+            plan.flux_attn_prefill(0, 0, q, k, v, 0, out)
+        torch.cuda.synchronize()
+        assert plan.flux_plan_status() == 0
+        i = np.arange(N, dtype=np.int64)
+        print(json.dumps({"profile_case": "prefill32k", "N": N, "launches": 2, "device_gb": 4 * q.numel() * 2 / 1e9 * 0.625,
+                          "flop_per_launch": 4 * w.n_q_heads * D * int((i + 1).sum())}))
     elif which == "heads":     # one dense, one sparse and one half-sparse-heads layer call at 256K tokens
         res = head_level_block(flux, dev, measured_peaks(), 1, reps=1)
         print(json.dumps({"profile_case": "heads", "launch_order": "each of dense, sparse, head-level: 3 warm-up + 1",
@@ -777,7 +806,7 @@ def main():
                     help="skip the other decode workloads (cfg4, cfg5) and the 128K prefill layers")
     ap.add_argument("--sustain-seconds", type=float, default=3.0,
                     help="after the K timed steps, keep replaying the step for this long and report the sustained rate")
-    ap.add_argument("--profile", default=None, choices=["decode", "prefill", "heads"],
+    ap.add_argument("--profile", default=None, choices=["decode", "decode_b1", "prefill", "prefill32k", "heads"],
                     help="run a small case of one kernel with few launches (for ncu captures) and exit")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -935,7 +964,7 @@ def main():
     per_launch_bytes = roof_bytes / max(kcnt, 1)
     per_launch_ms = kms / max(kcnt, 1)
     ach = per_launch_bytes / (per_launch_ms * 1e-3) / 1e9
-    tr = traffic_note("decode_kernel")
+    tr = traffic_note("decode_fused_kernel" if decode_kernel_name(flux, args.decode_kernel, w.batch).startswith("decode_fused") else "decode_kernel")
     roof = {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": ach / peaks["hbm_gbs"], "peak_source": peaks["source"] + " (copy bandwidth)",
             "kernel": decode_kernel_name(flux, args.decode_kernel, w.batch),

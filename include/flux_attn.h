@@ -342,14 +342,14 @@ int flux_attn_combine(flux_plan *plan, int32_t B, int32_t n_sets, const float *p
 int flux_plan_set_launch_overlap(flux_plan *plan, int32_t on);
 
 /* Which kernels flux_attn_decode / flux_attn_decode_step launch.  FLUX_DECODE_AUTO (the default)
- * runs the single-launch kernel for batches of at most 4 requests (the batch-1 latency setting of
- * Appendix C.3: one launch does the split-K attention and the merge, the CTA that finishes a
- * (request, KV head) last merges its partials) and the two-launch pair (split-K kernel + combine
- * pass) above that; the other two values force one of them.  FLUX_DECODE_SINGLE_LAUNCH is honoured
- * for batches of at most 8 requests and at most 64 KV heads, otherwise the pair runs.  Both compute
- * Eq. 1 / Eq. 2 over the same rows.  The single-launch kernel is issued with programmatic stream
- * serialisation: it starts with a grid-dependency wait, so results never depend on it, and it lets
- * the next such launch in the stream be set up while it drains. */
+ * runs the single-launch kernel for batches of at most 32 requests and at most 64 KV heads (one launch
+ * does the split-K attention and the merge: the CTA that finishes a (request, KV head) last merges its
+ * partials; it covers the batch-1 latency setting of Appendix C.3 and the batched workloads alike) and
+ * the two-launch pair (split-K kernel + combine pass) beyond that; the other two values force one of
+ * them where the shape allows.  Both compute Eq. 1 / Eq. 2 over the same rows.  The single-launch
+ * kernel is issued with programmatic stream serialisation: it starts with a grid-dependency wait (see
+ * flux_plan_set_launch_overlap), so results never depend on it, and it lets the next such launch in
+ * the stream be set up while it drains. */
 #define FLUX_DECODE_AUTO          0
 #define FLUX_DECODE_TWO_LAUNCH    1
 #define FLUX_DECODE_SINGLE_LAUNCH 2

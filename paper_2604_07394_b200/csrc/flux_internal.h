@@ -20,8 +20,8 @@ constexpr int kDecStages = 3;       // cp.async stages per warp
 constexpr int kDecStageBytes = kDecTile * kRowBytes * 2;  // K tile + V tile
 constexpr int kDecMaxCtas = 512;    // upper bound used to size the workspace
 constexpr int kMaxBatch = 1024;     // prefix tables live in shared memory
-constexpr int kDecFusedMaxBatch = 8;    // largest batch the single-launch decode kernel takes
-constexpr int kDecFusedAutoBatch = 4;   // largest batch it is chosen for by default
+constexpr int kDecFusedMaxBatch = 32;   // largest batch the single-launch decode kernel takes
+constexpr int kDecFusedAutoBatch = 32;  // largest batch it is chosen for by default
 constexpr int kDecFusedMaxKvHeads = 64;
 constexpr int kRouterMaxWidth = 4096;   // largest hidden width of the router MLPs (sizes the scratch)
 

@@ -51,7 +51,8 @@ constexpr int OFF_BAR = OFF_KV + kKvSlots * kTileBytes;
 //            Q_EMPTY   (hands the Q tiles over from one work item to the next)
 constexpr int BAR_Q_FULL = 0, BAR_KV_FULL = 1, BAR_KV_EMPTY = BAR_KV_FULL + kKvSlots,
               BAR_S_FULL = BAR_KV_EMPTY + kKvSlots, BAR_P_FULL = BAR_S_FULL + 2, BAR_O_FULL = BAR_P_FULL + 4,
-              BAR_Q_EMPTY = BAR_O_FULL + 2, kNumBars = BAR_Q_EMPTY + 1;
+              BAR_Q_EMPTY = BAR_O_FULL + 2, BAR_DRAIN = BAR_Q_EMPTY + 1,   // DRAIN: only used when a CTA gives up
+              kNumBars = BAR_DRAIN + 1;
 static_assert(kNumBars <= 24, "barrier area");
 constexpr int OFF_TMEM_PTR = OFF_BAR + 24 * 8;
 constexpr int OFF_ABORT = OFF_TMEM_PTR + 4;
@@ -227,15 +228,17 @@ struct TileWalk {
 // ================= TMA producer (one warp, one issuing lane) =================
 template <bool kBlock>
 __device__ __forceinline__ void role_load(Cta &c, const TcArgs &a, const CUtensorMap *tm_q, const CUtensorMap *tm_k,
-                                          const CUtensorMap *tm_v)
+                                          const CUtensorMap *tm_v, int &qi, int &q_armed)
 {
-    int qi = 0;                                      // K / V tiles requested so far (ring position)
+    // qi: K / V tiles requested so far (ring position); q_armed: items whose Q tiles have been requested.  Both are
+    // the caller's, so that a CTA that gives up knows which copies may still be on their way.
     for (int k = 0;; ++k) {
         const int item = item_of(k);
         if (item >= a.n_items) break;
         decode_item(a, item, c.fa, c);
         // Q of the next item may overwrite Q of this one once its last QK^T has completed
         if (k > 0 && !c.wait(BAR_Q_EMPTY, (uint32_t)((k - 1) & 1))) return;
+        q_armed = k + 1;
         if (elect_one()) {
             mbar_expect_tx(c.bar(BAR_Q_FULL), (uint32_t)(c.nslots * kTileBytes));
             for (int t = 0; t < c.nslots; ++t) {
@@ -547,6 +550,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
             mbar_init(c.bar(BAR_O_FULL + t), 1);
         }
         mbar_init(c.bar(BAR_Q_EMPTY), 1);
+        mbar_init(c.bar(BAR_DRAIN), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -561,10 +565,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     c.tmem = *tmem_ptr_smem;
 
     // Each warpgroup executes one setmaxnreg, all four of its warps the same one.
+    int kv_requested = 0, q_requested = 0;               // the producer warp's counters (see the teardown)
     if (warp >= 8) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
         if (warp == 8) {
-            role_load<kBlock>(c, a, &tm_q, &tm_k, &tm_v);
+            role_load<kBlock>(c, a, &tm_q, &tm_k, &tm_v, kv_requested, q_requested);
         } else if (warp == 9) {
             role_mma<kBlock>(c, a);
         }
@@ -577,8 +582,25 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constan
     tc_fence_before();
     __syncthreads();
     if (*c.abort_flag) {
-        // let copies and MMAs that were already issued land before the shared memory and TMEM go away
-        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+        // A wait gave up somewhere: copies and MMAs that were already issued must land before the shared memory and
+        // TMEM go away.  The producer waits for the last copy it requested into each ring slot and for the last Q
+        // tiles (their barriers complete when the bytes have arrived, whoever was to consume them); the issuer commits
+        // once more and waits for that commit, which follows every MMA it issued.  These waits are bounded too.
+        auto drain = [&](int bar, uint32_t parity) {
+            for (int i = 0; i < 200 && !mbar_try(c.bar(bar), parity); ++i) __nanosleep(1000);
+        };
+        if (warp == 8) {
+            for (int s = 0; s < kKvSlots; ++s) {
+                const int last = kv_requested - 1 - ((kv_requested - 1 - s) % kKvSlots + kKvSlots) % kKvSlots;   // latest request into slot s
+                if (kv_requested > 0 && last >= 0) drain(BAR_KV_FULL + s, (uint32_t)((last / kKvSlots) & 1));
+            }
+            if (q_requested > 0) drain(BAR_Q_FULL, (uint32_t)((q_requested - 1) & 1));
+        }
+        if (warp == 9) {
+            if (elect_one()) tc_commit(c.bar(BAR_DRAIN));
+            drain(BAR_DRAIN, 0u);
+        }
+        __syncthreads();
     }
     if (warp == 9) {
         tc_fence_after();

@@ -87,8 +87,9 @@ def test_prefill_256k_in_chunks_sampled_rows(flux):
     assert plan.flux_plan_status() == 0
 
 
-@pytest.mark.parametrize("cfg,dk", [("cfg3", 0), ("cfg3", 2), ("cfg4", 0), ("cfg4", 1), ("cfg4", 3), ("cfg5", 0)],
-                         ids=["cfg3", "cfg3_single_launch", "cfg4", "cfg4_two_launch", "cfg4_overlap", "cfg5"])
+@pytest.mark.parametrize("cfg,dk", [("cfg3", 0), ("cfg3", 1), ("cfg3", 3), ("cfg4", 0), ("cfg4", 1), ("cfg4", 3), ("cfg5", 1), ("cfg5", 3)],
+                         ids=["cfg3", "cfg3_two_launch", "cfg3_overlap", "cfg4", "cfg4_two_launch", "cfg4_overlap", "cfg5_two_launch",
+                              "cfg5_overlap"])
 def test_decode_full_size_sampled(flux, cfg, dk):
     """The decode workloads as bench.py builds them (compact sparse caches, per-request masks,
     ragged lengths for cfg5): two steps; at each, for every request two FA and two SA layers are

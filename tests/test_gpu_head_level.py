@@ -77,6 +77,7 @@ def test_uniform_head_masks_equal_the_layer_level_call(flux):
     Hq, Hkv, S, W, lens = 32, 8, 64, 192, [900, 257, 256, 40]
     B, cap = len(lens), 1024
     plan = flux.Plan(flux.make_config(2, Hq, Hkv, S, W, B, cap), DEV)
+    plan.flux_debug_decode_kernel(flux.FLUX_DECODE_TWO_LAUNCH)      # the kernels the head-level call runs
     plan.flux_router_apply(mask=np.array([[1, 0]] * B, dtype=np.uint8))
     kc, vc = _caches(flux, lens, Hkv, cap, 55)
     ktab, vtab = flux.pointer_table(kc, DEV), flux.pointer_table(vc, DEV)

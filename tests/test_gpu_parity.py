@@ -35,7 +35,7 @@ def _plan(flux, L, Hq, Hkv, S, W, B, max_ctx, layout=0, decode_kernel=None):
 
 
 # Both decode paths run every decode test: the two-launch pair (split-K kernel + combine pass) and the
-# single-launch kernel (taken for batches of at most 8 requests when forced; larger batches fall back
+# single-launch kernel (taken for batches of at most 32 requests when forced; larger batches fall back
 # to the pair, so those cases run the pair twice); the single-launch kernel also with launch overlap on
 # (schedule and first tile loads ahead of the grid-dependency wait: the calls these tests make keep the
 # promise that mode asks for).
@@ -201,7 +201,8 @@ DECODE_CASES = [
     (16, 16, 32, 64, [200, 97], 0),
     (28, 4, 16, 48, [20000], 0),                                   # batch 1: every CTA busy, several units each
     (28, 4, 128, 4096, [20000], 1),
-    (8, 8, 64, 128, [5000, 3, 129, 128, 127, 4097, 1, 700], 1),    # the largest batch the single-launch kernel takes
+    (8, 8, 64, 128, [5000, 3, 129, 128, 127, 4097, 1, 700], 1),    # a mixed batch of eight
+    (8, 2, 16, 48, [70 * (b % 5) + b for b in range(32)], 0),       # the largest batch the single-launch kernel takes (incl. an inactive request)
     (32, 2, 0, 300, [2500, 2500], 0),                              # 16 query heads per KV head (two merge passes)
 ]
 
