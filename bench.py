@@ -482,7 +482,9 @@ def prefill_block(flux, dev, peaks, warmup):
                            "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],
                            "frac_of_burst_peak": ach / peaks["bf16_tflops"],
                            "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
-                           "kernel": "FA prefill layer", "traffic": traffic_note("prefill_fa")}
+                           "kernel": "FA prefill layer",
+                           "traffic": (traffic_note("prefill_fa") or {}).get("dram_bytes_per_launch"),
+                           "traffic_source": (traffic_note("prefill_fa") or {}).get("source")}
     plan.close()
     return res
 
