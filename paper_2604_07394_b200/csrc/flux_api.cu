@@ -237,26 +237,52 @@ __global__ void kv_retain_kernel(const uint4 *__restrict__ k_src, const uint4 *_
 // K, V rows and its query rows straight from host memory, each byte once -- the K, V rows go into
 // the caches like kv_append_kernel does, the query rows into device staging (the decode kernel
 // re-reads them from every CTA, which must not cross the bus).
-__global__ void host_ingest_kernel(const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
-                                   const uint4 *__restrict__ q_host, uint4 *__restrict__ q_stage, int q_u4,
-                                   void *const *__restrict__ k_caches, void *const *__restrict__ v_caches,
-                                   const int32_t *__restrict__ pos, const uint8_t *__restrict__ mask,
-                                   int L, int layer, int row_u4, int S, int W, int layout,
-                                   int max_context, uint32_t *status)
+// Issued with programmatic stream serialisation when launch overlap is on: the reads from host memory (the slow part:
+// they cross the bus) are done before the grid-dependency wait, into registers, while the previous decode launch is
+// still running; everything the kernel writes -- the query staging that launch reads, the cache rows -- comes after it.
+constexpr int kIngestQ = 8, kIngestKV = 2;   // 16-byte pieces per thread held in registers across the wait
+__global__ void __launch_bounds__(256)
+host_ingest_kernel(const uint4 *__restrict__ k_new, const uint4 *__restrict__ v_new,
+                   const uint4 *__restrict__ q_host, uint4 *__restrict__ q_stage, int q_u4,
+                   void *const *__restrict__ k_caches, void *const *__restrict__ v_caches,
+                   const int32_t *__restrict__ pos, const uint8_t *__restrict__ mask,
+                   int L, int layer, int row_u4, int S, int W, int layout,
+                   int max_context, uint32_t *status)
 {
-    const int b = blockIdx.x;
-    for (int i = threadIdx.x; i < q_u4; i += blockDim.x) q_stage[(int64_t)b * q_u4 + i] = q_host[(int64_t)b * q_u4 + i];
+    asm volatile("griddepcontrol.launch_dependents;\n" ::: "memory");
+    const int b = blockIdx.x, tid = threadIdx.x, nt = blockDim.x;
+    uint4 qr[kIngestQ], kr[kIngestKV], vr[kIngestKV];
+#pragma unroll
+    for (int j = 0; j < kIngestQ; ++j)
+        if (tid + j * nt < q_u4) qr[j] = q_host[(int64_t)b * q_u4 + tid + j * nt];
+#pragma unroll
+    for (int j = 0; j < kIngestKV; ++j)
+        if (tid + j * nt < row_u4) {
+            kr[j] = k_new[(int64_t)b * row_u4 + tid + j * nt];
+            vr[j] = v_new[(int64_t)b * row_u4 + tid + j * nt];
+        }
     const int p = pos[b];
+    const bool compact = (layout == FLUX_KV_COMPACT_SA) && (mask[b * L + layer] == 0);
+    uint4 *kc = (uint4 *)k_caches[b], *vc = (uint4 *)v_caches[b];
+    asm volatile("griddepcontrol.wait;\n" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < kIngestQ; ++j)
+        if (tid + j * nt < q_u4) q_stage[(int64_t)b * q_u4 + tid + j * nt] = qr[j];
+    for (int i = tid + kIngestQ * nt; i < q_u4; i += nt) q_stage[(int64_t)b * q_u4 + i] = q_host[(int64_t)b * q_u4 + i];
     if (p < 0) return;
     if (p >= max_context) {
-        if (threadIdx.x == 0) atomicOr(status, FLUX_STATUS_BAD_LENGTH);
+        if (tid == 0) atomicOr(status, FLUX_STATUS_BAD_LENGTH);
         return;
     }
-    const bool compact = (layout == FLUX_KV_COMPACT_SA) && (mask[b * L + layer] == 0);
     const int64_t row = cache_row(p, compact, S, W);
-    uint4 *kd = (uint4 *)k_caches[b] + row * row_u4;
-    uint4 *vd = (uint4 *)v_caches[b] + row * row_u4;
-    for (int i = threadIdx.x; i < row_u4; i += blockDim.x) {
+    uint4 *kd = kc + row * row_u4, *vd = vc + row * row_u4;
+#pragma unroll
+    for (int j = 0; j < kIngestKV; ++j)
+        if (tid + j * nt < row_u4) {
+            kd[tid + j * nt] = kr[j];
+            vd[tid + j * nt] = vr[j];
+        }
+    for (int i = tid + kIngestKV * nt; i < row_u4; i += nt) {
         kd[i] = k_new[(int64_t)b * row_u4 + i];
         vd[i] = v_new[(int64_t)b * row_u4 + i];
     }
@@ -686,12 +712,21 @@ int flux_attn_decode_host(flux_plan *plan, int32_t layer, int32_t B, const void 
     void *mo = const_cast<void *>(mapped_host_ptr(out_host));
     if (mq && mk && mv && mo && aligned16(mq) && aligned16(mk) && aligned16(mv) && aligned16(mo)) {
         const int row_u4 = c.n_kv_heads * kRowBytes / 16;
-        host_ingest_kernel<<<B, 256, 0, st>>>((const uint4 *)mk, (const uint4 *)mv, (const uint4 *)mq, (uint4 *)dq,
-                                              c.n_q_heads * kRowBytes / 16, k_caches, v_caches, pos, plan->d_mask,
-                                              c.n_layers, layer, row_u4, c.sink, c.window, c.kv_layout,
-                                              c.max_context, (uint32_t *)(ws + plan->lay.status));
+        cudaLaunchConfig_t lc = {};
+        lc.gridDim = dim3((unsigned)B);
+        lc.blockDim = dim3(256);
+        lc.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        lc.attrs = attr;
+        lc.numAttrs = plan->launch_overlap ? 1 : 0;   // same promise as for the decode launch (flux_plan_set_launch_overlap)
+        rc = check_cuda(cudaLaunchKernelEx(&lc, host_ingest_kernel, (const uint4 *)mk, (const uint4 *)mv, (const uint4 *)mq,
+                                           (uint4 *)dq, c.n_q_heads * kRowBytes / 16, (void *const *)k_caches,
+                                           (void *const *)v_caches, pos, plan->d_mask, c.n_layers, layer, row_u4, c.sink,
+                                           c.window, c.kv_layout, c.max_context, (uint32_t *)(ws + plan->lay.status)),
+                        "host ingest kernel launch");
         plan->launches++;
-        rc = check_cuda(cudaGetLastError(), "host ingest kernel launch");
         if (!rc)
             rc = launch_decode(plan, layer, B, dq, (const void *const *)k_caches, (const void *const *)v_caches,
                                ctx_len, mo, st);

@@ -434,12 +434,15 @@ def test_fused_decode_step_equals_append_then_decode(flux, layout, dk):
     assert plan.flux_plan_status() == 0
 
 
+@DECODE_KERNELS
 @pytest.mark.parametrize("pinned", [True, False], ids=["pinned_zero_copy", "pageable_staged"])
-def test_decode_host_entry_point_matches_device_entry_point(flux, pinned):
+def test_decode_host_entry_point_matches_device_entry_point(flux, pinned, dk):
+    """Host buffers in, host buffers out, two layers back to back (with launch overlap the second layer's ingest
+    kernel reads its host inputs while the first layer's decode launch is still running)."""
     pin = (lambda t: t.pin_memory()) if pinned else (lambda t: t)
     Hq, Hkv, S, W, B, L = 8, 2, 4, 8, 3, 2
     lens = [30, 9, 17]
-    plan = _plan(flux, L, Hq, Hkv, S, W, B, 64)
+    plan = _plan(flux, L, Hq, Hkv, S, W, B, 64, 0, dk)
     plan.flux_router_apply(mask=np.array([[1, 0], [0, 0], [1, 1]], dtype=np.uint8))
     kc = [synth.normal_bf16((64, Hkv, 128), 5, b, DEV) for b in range(B)]
     vc = [synth.normal_bf16((64, Hkv, 128), 6, b, DEV) for b in range(B)]
@@ -449,15 +452,18 @@ def test_decode_host_entry_point_matches_device_entry_point(flux, pinned):
     vn = pin(synth.normal_bf16((B, Hkv, 128), 7, 2, "cpu"))
     pos = torch.tensor([n - 1 for n in lens], dtype=torch.int32, device=DEV)
     ctx = torch.tensor(lens, dtype=torch.int32, device=DEV)
-    out_h = pin(torch.empty((B, Hq, 128), dtype=torch.bfloat16))
+    out_h = [pin(torch.empty((B, Hq, 128), dtype=torch.bfloat16)) for _ in range(L)]
+    kt, vt = flux.pointer_table(kc, DEV), flux.pointer_table(vc, DEV)
+    for rep in range(3):                                 # the layers' calls back to back, nothing in between
+        for layer in range(L):
+            plan.flux_attn_decode_host(layer, B, q, kn, vn, kt, vt, pos, ctx, out_h[layer])
+    torch.cuda.synchronize()
+    kt2, vt2 = flux.pointer_table(kc2, DEV), flux.pointer_table(vc2, DEV)
     for layer in range(L):
-        kt, vt = flux.pointer_table(kc, DEV), flux.pointer_table(vc, DEV)
-        plan.flux_attn_decode_host(layer, B, q, kn, vn, kt, vt, pos, ctx, out_h)
-        torch.cuda.synchronize()
-        kt2, vt2 = flux.pointer_table(kc2, DEV), flux.pointer_table(vc2, DEV)
         plan.flux_kv_append(layer, B, kn.to(DEV), vn.to(DEV), kt2, vt2, pos)
         out_d = plan.flux_attn_decode(layer, B, q.to(DEV), kt2, vt2, ctx)
-        assert torch.equal(out_d.cpu(), out_h)
+        assert torch.equal(out_d.cpu(), out_h[layer]), layer
+    assert plan.flux_plan_status() == 0
 
 
 def test_decode_at_the_maximum_batch_and_group_size(flux):
