@@ -483,6 +483,7 @@ int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *con
     a.touch_words = p->touch_words;
     a.head_mask = head_mask;
     a.tickets = (uint32_t *)(ws + p->lay.tickets);
+    a.done = a.tickets + (size_t)kDecFusedMaxBatch * c.n_kv_heads;
     a.overlap = (p->launch_overlap && p->touch == nullptr) ? 1 : 0;   // the debug bitmap is written by the loaders
     a.key_begin = part ? part->key_begin : nullptr;
     a.key_end = part ? part->key_end : nullptr;
@@ -643,6 +644,7 @@ extern "C" int flux_attn_decode_noalloc(const flux_config *cfg, int32_t layer, i
     a.touch_words = 0;
     a.head_mask = nullptr;
     a.tickets = nullptr;
+    a.done = nullptr;
     a.overlap = 0;
     a.key_begin = a.key_end = nullptr;
     a.pout_o = a.pout_ml = nullptr;

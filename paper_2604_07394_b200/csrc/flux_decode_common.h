@@ -33,8 +33,10 @@ struct DecArgs {
     // head-level comparison mode (flux_attn_decode_heads): uint8 [B][Hkv], 1 = the KV head's group
     // attends densely, 0 = sink + window; NULL in the routed (layer-level) calls
     const uint8_t *head_mask;
-    // arrival counters of the single-launch kernel, one per (request, KV head); zero between launches
+    // single-launch kernel: per (request, KV head) the count of CTAs that have announced their partials, and the
+    // count of CTAs that have started merging them; both zero between launches
     uint32_t *tickets;
+    uint32_t *done;
     // single-launch kernel only: schedule and first tile loads before the grid-dependency wait
     int overlap;
     // partial evaluation over a key range (flux_attn_decode_partial): positions [key_begin[b], key_end[b]) of each

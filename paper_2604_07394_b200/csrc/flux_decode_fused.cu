@@ -9,10 +9,15 @@
 //    heads of one KV head only (a quarter or an eighth of what a whole-row CTA would write);
 //  * when a CTA leaves a (request, KV head) segment its eight warps merge their flash-attention
 //    states through shared memory into one partial (O, m, l) per query head;
-//  * the CTA then takes a ticket on the segment's arrival counter; the CTA that draws the last
-//    ticket merges the segment's partials (Eq. 1 / Eq. 2 are sums over disjoint key sets, which
-//    merge by rescaling with 2^(m_p - m)) and writes the bf16 output rows.  Nobody waits: every
-//    CTA but the last simply leaves.
+//  * the CTA then announces itself on the segment's arrival counter and goes on; a CTA that covers a
+//    whole segment alone writes the output rows straight away instead;
+//  * when a CTA has finished all its tiles it takes its share of the merging: the i-th CTA of a
+//    segment merges query head i (and i + the number of the segment's CTAs, ...) of that segment: it
+//    waits -- a bounded spin on the arrival counter, which only CTAs of this same launch advance, none
+//    of which waits for anything before announcing itself -- until all the segment's CTAs have announced
+//    themselves, copies the head's partials into its idle stage memory and merges them (Eq. 1 / Eq. 2 are
+//    sums over disjoint key sets, which merge by rescaling with 2^(m_p - m)).  The merge of a segment is
+//    thus spread over as many SMs as it has query heads, each reading a seventh (G = 7) of the partials.
 //
 // The launch is issued with programmatic stream serialisation and releases its dependents at once, so
 // the next launch of this kind is set up while this one drains.  By default the kernel waits for the
@@ -35,6 +40,8 @@ constexpr int kFuMergeMlBytes = kDecWarps * kFuRows * 2 * (int)sizeof(float);
 constexpr int kFuSmemBytes = kFuStageBytes + kFuMergeOBytes + kFuMergeMlBytes;
 // partial rows (512 bytes of O and 8 bytes of (m, l) each) the idle stage memory takes for the last CTA's merge
 constexpr int kFuStagedRows = kFuStageBytes / (kHeadDim * 4 + 8);
+constexpr long long kFuWaitCycles = 2000000000ll;   // bound of the wait for a segment's arrivals (about a second)
+constexpr int kFuMaxDuties = 2;                      // segments a CTA shares with other CTAs: the first and the last of its span
 
 struct FuIt {
     int u;      // global unit index
@@ -88,9 +95,16 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
     __shared__ int s_mode[kDecFusedMaxBatch];
     __shared__ const unsigned char *s_k[kDecFusedMaxBatch];
     __shared__ const unsigned char *s_v[kDecFusedMaxBatch];
-    __shared__ unsigned s_ticket;
+    __shared__ int s_duty[kFuMaxDuties][5];   // segment, first CTA, CTAs, request, KV head of the segments to help merge
+    __shared__ int s_n_duty;
+    __shared__ int s_abort;
+    __shared__ unsigned s_order;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        s_n_duty = 0;
+        s_abort = 0;
+    }
     float *mo = reinterpret_cast<float *>(smem + kFuStageBytes);
     float *mml = reinterpret_cast<float *>(smem + kFuStageBytes + kFuMergeOBytes);
 
@@ -248,9 +262,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
     // Leaves a segment: CTA-level merge of the eight warps' states, one partial per query head to
     // global memory, a ticket; the last CTA of the segment merges all partials and writes the output.
     // Every warp of the CTA calls this at the same unit (the iterators do not depend on the warp).
-    // `idle`: no tile loads are in flight any more (the CTA's last segment), so the stage memory can
-    // take the partials.
-    auto flush = [&](const bool idle) {
+    auto flush = [&]() {
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             l_r[i] += __shfl_xor_sync(0xffffffffu, l_r[i], 1);
@@ -276,150 +288,31 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
             if (warp < rows) {
                 float m, l;
                 const float4 acc = fu_merge_row(mo, mml, warp, lane, m, l);
-                const size_t e = my_slot * a.G + pass * kFuRows + warp;
-                *reinterpret_cast<float4 *>(a.part_o + e * kHeadDim + lane * 4) = acc;
-                if (lane == 0) *reinterpret_cast<float2 *>(a.part_ml + e * 2) = make_float2(m, l);
-            }
-            if (pass + 1 < passes) __syncthreads();   // the buffer is reused; after the last pass the ticket barrier does it
-        }
-        // One release-acquire ticket per CTA: the CTA's partial stores (ordered before thread 0 by the barrier)
-        // become visible before the ticket is, and whoever draws the last ticket sees every partial.
-        __syncthreads();
-        if (tid == 0) {
-            unsigned ticket;
-            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;\n" : "=r"(ticket) : "l"(a.tickets + cur_seg) : "memory");
-            s_ticket = ticket;
-        }
-        __syncthreads();
-        if (s_ticket != (unsigned)(n_part - 1)) return;
-        // ---- last CTA of the segment ----------------------------------------------------------------
-        // The segment's partials are one contiguous block: n_part * G rows from entry (c_first + cur_seg) * G.
-        const size_t e_base = ((size_t)c_first + cur_seg) * a.G;
-        const int n_rows = n_part * a.G;
-        float2 *s_ml = reinterpret_cast<float2 *>(mml);
-        const float *so = reinterpret_cast<const float *>(smem);
-        if (idle && n_rows <= kFuStagedRows) {
-            // No tile loads are in flight (the CTA's last segment): the block comes into the stage memory by one
-            // round of asynchronous copies; then one warp per query head: weights 2^(m_p - m) first (lanes over
-            // the partials), then the weighted sum with four partials in flight.  The loops stay rolled: this
-            // code runs once per launch, and its size costs more than its arithmetic.
-            float2 *st_ml = reinterpret_cast<float2 *>(smem + (size_t)kFuStagedRows * kHeadDim * 4);
-            const unsigned char *src = reinterpret_cast<const unsigned char *>(a.part_o + e_base * kHeadDim);
-            const uint32_t dst = smem_u32(smem);
-            for (int c = tid; c < n_rows * (kHeadDim * 4 / 16); c += blockDim.x) cp_async16(dst + c * 16, src + (size_t)c * 16, 16);
-            cp_async_commit();
-            for (int i = tid; i < n_rows; i += blockDim.x) st_ml[i] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + (e_base + i) * 2));
-            cp_async_wait<0>();
-            __syncthreads();
-            for (int r = warp; r < a.G; r += kDecWarps) {
-                float m = kNegBig;
-                for (int p = lane; p < n_part; p += 32) m = fmaxf(m, st_ml[p * a.G + r].x);
-#pragma unroll
-                for (int d = 16; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
-                float l = 0.f;
-                for (int p = lane; p < n_part; p += 32) {
-                    const float2 ml = st_ml[p * a.G + r];
-                    const float w = fast_exp2(ml.x - m);
-                    st_ml[p * a.G + r].x = w;
-                    l += ml.y * w;
-                }
-#pragma unroll
-                for (int d = 16; d >= 1; d >>= 1) l += __shfl_xor_sync(0xffffffffu, l, d);
-                __syncwarp();
-                float4 acc[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                const float *row0 = so + (size_t)r * kHeadDim + lane * 4;
-                const float2 *w0 = st_ml + r;
-                int p = 0;
-#pragma unroll 1
-                for (; p + 4 <= n_part; p += 4) {
-#pragma unroll
-                    for (int u = 0; u < 4; ++u) {
-                        const float w = w0[(p + u) * a.G].x;
-                        const float4 v = *reinterpret_cast<const float4 *>(row0 + (size_t)(p + u) * a.G * kHeadDim);
-                        acc[u].x += v.x * w;
-                        acc[u].y += v.y * w;
-                        acc[u].z += v.z * w;
-                        acc[u].w += v.w * w;
-                    }
-                }
-#pragma unroll 1
-                for (; p < n_part; ++p) {
-                    const float w = w0[p * a.G].x;
-                    const float4 v = *reinterpret_cast<const float4 *>(row0 + (size_t)p * a.G * kHeadDim);
-                    acc[0].x += v.x * w;
-                    acc[0].y += v.y * w;
-                    acc[0].z += v.z * w;
-                    acc[0].w += v.w * w;
-                }
-                const float inv = l > 0.f ? 1.0f / l : 0.f;
-                uint2 pk;
-                pk.x = pack_bf16((acc[0].x + acc[1].x + acc[2].x + acc[3].x) * inv, (acc[0].y + acc[1].y + acc[2].y + acc[3].y) * inv);
-                pk.y = pack_bf16((acc[0].z + acc[1].z + acc[2].z + acc[3].z) * inv, (acc[0].w + acc[1].w + acc[2].w + acc[3].w) * inv);
-                *reinterpret_cast<uint2 *>(a.out + ((size_t)seg_b * a.Hq + (size_t)seg_head * a.G + r) * kHeadDim + lane * 4) = pk;
-            }
-        } else {
-            // Tile loads of the next segment are in flight (or the block is too large for the stage memory): warp w
-            // folds partials w, w + 8, ... for every query head straight from global memory, then the eight warps'
-            // results are merged like the per-CTA states above.
-            for (int pass = 0; pass < passes; ++pass) {
-                const int rows = min(a.G - pass * kFuRows, kFuRows);
-                float4 acc[kFuRows];
-                float mm[kFuRows], ll[kFuRows];
-#pragma unroll
-                for (int r = 0; r < kFuRows; ++r) {
-                    acc[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    mm[r] = kNegBig;
-                    ll[r] = 0.f;
-                }
-#pragma unroll 1
-                for (int p = warp; p < n_part; p += kDecWarps) {
-                    const size_t e0 = e_base + (size_t)p * a.G + pass * kFuRows;
-                    float2 ml[kFuRows];
-                    float4 v[kFuRows];
-#pragma unroll
-                    for (int r = 0; r < kFuRows; ++r) {
-                        if (r < rows) {
-                            ml[r] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + (e0 + r) * 2));
-                            v[r] = __ldcg(reinterpret_cast<const float4 *>(a.part_o + (e0 + r) * kHeadDim + lane * 4));
-                        } else {
-                            ml[r] = make_float2(kNegBig, 0.f);
-                            v[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        }
-                    }
-#pragma unroll
-                    for (int r = 0; r < kFuRows; ++r) {
-                        const float m_new = fmaxf(mm[r], ml[r].x);
-                        const float sc = fast_exp2(mm[r] - m_new), sp = fast_exp2(ml[r].x - m_new);
-                        acc[r].x = acc[r].x * sc + v[r].x * sp;
-                        acc[r].y = acc[r].y * sc + v[r].y * sp;
-                        acc[r].z = acc[r].z * sc + v[r].z * sp;
-                        acc[r].w = acc[r].w * sc + v[r].w * sp;
-                        ll[r] = ll[r] * sc + ml[r].y * sp;
-                        mm[r] = m_new;
-                    }
-                }
-#pragma unroll
-                for (int r = 0; r < kFuRows; ++r) {
-                    *reinterpret_cast<float4 *>(mo + (warp * kFuRows + r) * kFuRowStride + lane * 4) = acc[r];
-                    if (lane == 0) s_ml[warp * kFuRows + r] = make_float2(mm[r], ll[r]);
-                }
-                __syncthreads();
-                if (warp < rows) {
-                    float m, l;
-                    const float4 s4 = fu_merge_row(mo, mml, warp, lane, m, l);
+                if (n_part == 1) {   // this CTA has the whole segment: the output row itself
                     const float inv = l > 0.f ? 1.0f / l : 0.f;
                     uint2 pk;
-                    pk.x = pack_bf16(s4.x * inv, s4.y * inv);
-                    pk.y = pack_bf16(s4.z * inv, s4.w * inv);
+                    pk.x = pack_bf16(acc.x * inv, acc.y * inv);
+                    pk.y = pack_bf16(acc.z * inv, acc.w * inv);
                     *reinterpret_cast<uint2 *>(a.out + ((size_t)seg_b * a.Hq + (size_t)seg_head * a.G + pass * kFuRows + warp) * kHeadDim +
                                                lane * 4) = pk;
+                } else {
+                    const size_t e = my_slot * a.G + pass * kFuRows + warp;
+                    *reinterpret_cast<float4 *>(a.part_o + e * kHeadDim + lane * 4) = acc;
+                    if (lane == 0) *reinterpret_cast<float2 *>(a.part_ml + e * 2) = make_float2(m, l);
                 }
-                __syncthreads();
             }
+            if (pass + 1 < passes || n_part == 1) __syncthreads();   // the buffer is reused (else the barrier below does it)
         }
-        if (tid == 0) a.tickets[cur_seg] = 0u;   // ready for the next launch (stream order)
+        if (n_part == 1) return;
+        // the CTA's partial stores (ordered before thread 0 by the barrier) become visible before its arrival is
+        __syncthreads();
+        if (tid == 0) {
+            asm volatile("red.release.gpu.global.add.u32 [%0], 1;\n" ::"l"(a.tickets + cur_seg) : "memory");
+            const int d = s_n_duty;       // at most two segments of a span are shared with other CTAs
+            s_duty[d][0] = cur_seg; s_duty[d][1] = c_first; s_duty[d][2] = n_part; s_duty[d][3] = seg_b; s_duty[d][4] = seg_head;
+            s_n_duty = d + 1;
+        }
+        __syncthreads();
     };
 
     // Query rows of a segment: 16 rows of 256 bytes (rows >= G zero-filled) into this warp's part of the merge
@@ -490,7 +383,7 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
         cp_async_wait<kDecStages - 1>();
         __syncwarp();
         if (cit.b * a.Hkv + cit.head != cur_seg) {
-            flush(false);
+            flush();
             enter_segment(cit);
             cp_async_wait<0>();
             __syncwarp();
@@ -509,8 +402,101 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
         }
     }
     cp_async_wait<0>();
-    __syncthreads();   // every warp is done with its stage memory
-    flush(true);
+    flush();
+    __syncthreads();   // every warp is done with its stage memory and the merge buffers
+
+    // ---- this CTA's share of the merging ---------------------------------------------------------------
+    const int n_duty = s_n_duty;
+    for (int d = 0; d < n_duty; ++d) {
+        const int seg = s_duty[d][0], c_first = s_duty[d][1], n_part = s_duty[d][2], db = s_duty[d][3], dh = s_duty[d][4];
+        const int idx = (int)blockIdx.x - c_first;       // this CTA's place among the segment's CTAs
+        if (idx >= a.G) continue;                        // more CTAs than query heads: the later ones have nothing to merge
+        // Wait until every CTA of the segment has announced itself (they all do, unconditionally, when they leave the
+        // segment).  The order in which the helpers get here decides who puts the counters back to zero: the last one,
+        // which knows that nobody will look at them again.
+        if (tid == 0) {
+            const long long t0 = clock64();
+            unsigned seen;
+            do {
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(seen) : "l"(a.tickets + seg) : "memory");
+                if (seen < (unsigned)n_part && clock64() - t0 > kFuWaitCycles) {
+                    atomicOr(a.status, FLUX_STATUS_WAIT_EXPIRED);
+                    s_abort = 1;
+                    break;
+                }
+            } while (seen < (unsigned)n_part);
+            unsigned order;
+            asm volatile("atom.relaxed.gpu.global.add.u32 %0, [%1], 1;\n" : "=r"(order) : "l"(a.done + seg) : "memory");
+            s_order = order;
+        }
+        __syncthreads();
+        if (s_abort) return;
+        const size_t e_base = ((size_t)c_first + seg) * a.G;      // partial p of query head r: entry e_base + p * G + r
+        float *st_o = reinterpret_cast<float *>(smem);
+        float2 *st_ml = reinterpret_cast<float2 *>(smem + (size_t)kFuStagedRows * kHeadDim * 4);
+        for (int r = idx; r < a.G; r += n_part) {
+            for (int p0 = 0; p0 < n_part; p0 += kFuStagedRows) {     // (one round unless a head has hundreds of partials)
+                const int np = min(n_part - p0, kFuStagedRows);
+                for (int c = tid; c < np * 32; c += blockDim.x) {
+                    const int p = c >> 5, piece = c & 31;
+                    cp_async16(smem_u32(st_o) + (uint32_t)c * 16u, a.part_o + (e_base + (size_t)(p0 + p) * a.G + r) * kHeadDim + piece * 4, 16);
+                }
+                cp_async_commit();
+                for (int p = tid; p < np; p += blockDim.x)
+                    st_ml[p] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + (e_base + (size_t)(p0 + p) * a.G + r) * 2));
+                cp_async_wait<0>();
+                __syncthreads();
+                // warp w folds partials w, w + 8, ... ; the warps' results go through the merge buffers; a later round
+                // of the same head starts from the merged state of the rounds before (kept by warp 0)
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                float m = kNegBig, l = 0.f;
+                if (p0 > 0 && warp == 0) {
+                    acc = *reinterpret_cast<const float4 *>(mo + (size_t)kDecWarps * kFuRows * kFuRowStride - kHeadDim + lane * 4);
+                    m = mml[kDecWarps * kFuRows * 2 - 2];
+                    l = mml[kDecWarps * kFuRows * 2 - 1];
+                }
+#pragma unroll 2
+                for (int p = warp; p < np; p += kDecWarps) {
+                    const float2 ml = st_ml[p];
+                    const float4 v = *reinterpret_cast<const float4 *>(st_o + (size_t)p * kHeadDim + lane * 4);
+                    const float m_new = fmaxf(m, ml.x);
+                    const float sc = fast_exp2(m - m_new), sp = fast_exp2(ml.x - m_new);
+                    acc.x = acc.x * sc + v.x * sp;
+                    acc.y = acc.y * sc + v.y * sp;
+                    acc.z = acc.z * sc + v.z * sp;
+                    acc.w = acc.w * sc + v.w * sp;
+                    l = l * sc + ml.y * sp;
+                    m = m_new;
+                }
+                *reinterpret_cast<float4 *>(mo + (warp * kFuRows) * kFuRowStride + lane * 4) = acc;
+                if (lane == 0) *reinterpret_cast<float2 *>(mml + (warp * kFuRows) * 2) = make_float2(m, l);
+                __syncthreads();
+                if (warp == 0) {
+                    float mm, ll;
+                    const float4 s4 = fu_merge_row(mo, mml, 0, lane, mm, ll);
+                    if (p0 + np < n_part) {          // more rounds to come: keep the state at the end of the buffers
+                        *reinterpret_cast<float4 *>(mo + (size_t)kDecWarps * kFuRows * kFuRowStride - kHeadDim + lane * 4) = s4;
+                        if (lane == 0) {
+                            mml[kDecWarps * kFuRows * 2 - 2] = mm;
+                            mml[kDecWarps * kFuRows * 2 - 1] = ll;
+                        }
+                    } else {
+                        const float inv = ll > 0.f ? 1.0f / ll : 0.f;
+                        uint2 pk;
+                        pk.x = pack_bf16(s4.x * inv, s4.y * inv);
+                        pk.y = pack_bf16(s4.z * inv, s4.w * inv);
+                        *reinterpret_cast<uint2 *>(a.out + ((size_t)db * a.Hq + (size_t)dh * a.G + r) * kHeadDim + lane * 4) = pk;
+                    }
+                }
+                __syncthreads();
+            }
+        }
+        const int helpers = n_part < a.G ? n_part : a.G;
+        if (tid == 0 && s_order == (unsigned)(helpers - 1)) {   // ready for the next launch (stream order)
+            a.tickets[seg] = 0u;
+            a.done[seg] = 0u;
+        }
+    }
 }
 
 }  // namespace

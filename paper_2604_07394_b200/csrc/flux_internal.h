@@ -40,7 +40,7 @@ struct WorkspaceLayout {
     size_t host_o;       // bf16  [max_batch][Hq][D]
     size_t router;       // fp32  [2*Hq*D + 3*kRouterMaxWidth] pooled descriptor and hidden activations
     size_t router_sync;  // uint32 [4] barrier counters and ticket of the one-launch router front end (zero between launches)
-    size_t tickets;      // uint32 [kDecFusedMaxBatch][Hkv] arrival counters of the single-launch decode (zero between launches)
+    size_t tickets;      // uint32 [2][kDecFusedMaxBatch][Hkv] arrival / helper counters of the single-launch decode (zero between launches)
     size_t total;
     int64_t slots;
 };
