@@ -98,7 +98,6 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
     __shared__ int s_duty[kFuMaxDuties][5];   // segment, first CTA, CTAs, request, KV head of the segments to help merge
     __shared__ int s_n_duty;
     __shared__ int s_abort;
-    __shared__ unsigned s_order;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -249,6 +248,98 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
             }
         }
     }
+    // Merges query heads r_first, r_first + r_step, ... of a segment whose partials come from n_part CTAs (c_first ...):
+    // waits until all of them have announced themselves, brings a head's partials into the stage memory (idle by then),
+    // folds them, writes the output row.  `helpers` CTAs do this for the segment; the last of them to get here puts
+    // the counters back to zero.  False when the wait ran out.
+    auto help = [&](int seg, int c_first, int n_part, int db, int dh, int r_first, int r_step, int helpers) -> bool {
+        // Wait until every CTA of the segment has announced itself (they all do, unconditionally, when they leave the
+        // segment).  The order in which the helpers get here decides who puts the counters back to zero: the last one,
+        // which knows that nobody will look at them again.
+        unsigned order = 0;
+        if (tid == 0) {
+            const long long t0 = clock64();
+            unsigned seen;
+            do {
+                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(seen) : "l"(a.tickets + seg) : "memory");
+                if (seen < (unsigned)n_part && clock64() - t0 > kFuWaitCycles) {
+                    atomicOr(a.status, FLUX_STATUS_WAIT_EXPIRED);
+                    s_abort = 1;
+                    break;
+                }
+            } while (seen < (unsigned)n_part);
+            // (the answer is needed only at the very end: nothing waits for this round trip)
+            asm volatile("atom.relaxed.gpu.global.add.u32 %0, [%1], 1;\n" : "=r"(order) : "l"(a.done + seg) : "memory");
+        }
+        __syncthreads();
+        if (s_abort) return false;
+        const size_t e_base = ((size_t)c_first + seg) * a.G;      // partial p of query head r: entry e_base + p * G + r
+        float *st_o = reinterpret_cast<float *>(smem);
+        float2 *st_ml = reinterpret_cast<float2 *>(smem + (size_t)kFuStagedRows * kHeadDim * 4);
+        for (int r = r_first; r < a.G; r += r_step) {
+            for (int p0 = 0; p0 < n_part; p0 += kFuStagedRows) {     // (one round unless a head has hundreds of partials)
+                const int np = min(n_part - p0, kFuStagedRows);
+                for (int c = tid; c < np * 32; c += blockDim.x) {
+                    const int p = c >> 5, piece = c & 31;
+                    cp_async16(smem_u32(st_o) + (uint32_t)c * 16u, a.part_o + (e_base + (size_t)(p0 + p) * a.G + r) * kHeadDim + piece * 4, 16);
+                }
+                cp_async_commit();
+                for (int p = tid; p < np; p += blockDim.x)
+                    st_ml[p] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + (e_base + (size_t)(p0 + p) * a.G + r) * 2));
+                cp_async_wait<0>();
+                __syncthreads();
+                // warp w folds partials w, w + 8, ... ; the warps' results go through the merge buffers; a later round
+                // of the same head starts from the merged state of the rounds before (kept by warp 0)
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                float m = kNegBig, l = 0.f;
+                if (p0 > 0 && warp == 0) {
+                    acc = *reinterpret_cast<const float4 *>(mo + (size_t)kDecWarps * kFuRows * kFuRowStride - kHeadDim + lane * 4);
+                    m = mml[kDecWarps * kFuRows * 2 - 2];
+                    l = mml[kDecWarps * kFuRows * 2 - 1];
+                }
+#pragma unroll 2
+                for (int p = warp; p < np; p += kDecWarps) {
+                    const float2 ml = st_ml[p];
+                    const float4 v = *reinterpret_cast<const float4 *>(st_o + (size_t)p * kHeadDim + lane * 4);
+                    const float m_new = fmaxf(m, ml.x);
+                    const float sc = fast_exp2(m - m_new), sp = fast_exp2(ml.x - m_new);
+                    acc.x = acc.x * sc + v.x * sp;
+                    acc.y = acc.y * sc + v.y * sp;
+                    acc.z = acc.z * sc + v.z * sp;
+                    acc.w = acc.w * sc + v.w * sp;
+                    l = l * sc + ml.y * sp;
+                    m = m_new;
+                }
+                *reinterpret_cast<float4 *>(mo + (warp * kFuRows) * kFuRowStride + lane * 4) = acc;
+                if (lane == 0) *reinterpret_cast<float2 *>(mml + (warp * kFuRows) * 2) = make_float2(m, l);
+                __syncthreads();
+                if (warp == 0) {
+                    float mm, ll;
+                    const float4 s4 = fu_merge_row(mo, mml, 0, lane, mm, ll);
+                    if (p0 + np < n_part) {          // more rounds to come: keep the state at the end of the buffers
+                        *reinterpret_cast<float4 *>(mo + (size_t)kDecWarps * kFuRows * kFuRowStride - kHeadDim + lane * 4) = s4;
+                        if (lane == 0) {
+                            mml[kDecWarps * kFuRows * 2 - 2] = mm;
+                            mml[kDecWarps * kFuRows * 2 - 1] = ll;
+                        }
+                    } else {
+                        const float inv = ll > 0.f ? 1.0f / ll : 0.f;
+                        uint2 pk;
+                        pk.x = pack_bf16(s4.x * inv, s4.y * inv);
+                        pk.y = pack_bf16(s4.z * inv, s4.w * inv);
+                        *reinterpret_cast<uint2 *>(a.out + ((size_t)db * a.Hq + (size_t)dh * a.G + r) * kHeadDim + lane * 4) = pk;
+                    }
+                }
+                __syncthreads();
+            }
+        }
+        if (tid == 0 && order == (unsigned)(helpers - 1)) {   // ready for the next launch (stream order)
+            a.tickets[seg] = 0u;
+            a.done[seg] = 0u;
+        }
+        return true;
+    };
+
     if (n_units == 0) return;
 
     // consumer state
@@ -408,94 +499,10 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_fused_kernel(DecArgs
     // ---- this CTA's share of the merging ---------------------------------------------------------------
     const int n_duty = s_n_duty;
     for (int d = 0; d < n_duty; ++d) {
-        const int seg = s_duty[d][0], c_first = s_duty[d][1], n_part = s_duty[d][2], db = s_duty[d][3], dh = s_duty[d][4];
+        const int c_first = s_duty[d][1], n_part = s_duty[d][2];
         const int idx = (int)blockIdx.x - c_first;       // this CTA's place among the segment's CTAs
         if (idx >= a.G) continue;                        // more CTAs than query heads: the later ones have nothing to merge
-        // Wait until every CTA of the segment has announced itself (they all do, unconditionally, when they leave the
-        // segment).  The order in which the helpers get here decides who puts the counters back to zero: the last one,
-        // which knows that nobody will look at them again.
-        if (tid == 0) {
-            const long long t0 = clock64();
-            unsigned seen;
-            do {
-                asm volatile("ld.acquire.gpu.global.u32 %0, [%1];\n" : "=r"(seen) : "l"(a.tickets + seg) : "memory");
-                if (seen < (unsigned)n_part && clock64() - t0 > kFuWaitCycles) {
-                    atomicOr(a.status, FLUX_STATUS_WAIT_EXPIRED);
-                    s_abort = 1;
-                    break;
-                }
-            } while (seen < (unsigned)n_part);
-            unsigned order;
-            asm volatile("atom.relaxed.gpu.global.add.u32 %0, [%1], 1;\n" : "=r"(order) : "l"(a.done + seg) : "memory");
-            s_order = order;
-        }
-        __syncthreads();
-        if (s_abort) return;
-        const size_t e_base = ((size_t)c_first + seg) * a.G;      // partial p of query head r: entry e_base + p * G + r
-        float *st_o = reinterpret_cast<float *>(smem);
-        float2 *st_ml = reinterpret_cast<float2 *>(smem + (size_t)kFuStagedRows * kHeadDim * 4);
-        for (int r = idx; r < a.G; r += n_part) {
-            for (int p0 = 0; p0 < n_part; p0 += kFuStagedRows) {     // (one round unless a head has hundreds of partials)
-                const int np = min(n_part - p0, kFuStagedRows);
-                for (int c = tid; c < np * 32; c += blockDim.x) {
-                    const int p = c >> 5, piece = c & 31;
-                    cp_async16(smem_u32(st_o) + (uint32_t)c * 16u, a.part_o + (e_base + (size_t)(p0 + p) * a.G + r) * kHeadDim + piece * 4, 16);
-                }
-                cp_async_commit();
-                for (int p = tid; p < np; p += blockDim.x)
-                    st_ml[p] = __ldcg(reinterpret_cast<const float2 *>(a.part_ml + (e_base + (size_t)(p0 + p) * a.G + r) * 2));
-                cp_async_wait<0>();
-                __syncthreads();
-                // warp w folds partials w, w + 8, ... ; the warps' results go through the merge buffers; a later round
-                // of the same head starts from the merged state of the rounds before (kept by warp 0)
-                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                float m = kNegBig, l = 0.f;
-                if (p0 > 0 && warp == 0) {
-                    acc = *reinterpret_cast<const float4 *>(mo + (size_t)kDecWarps * kFuRows * kFuRowStride - kHeadDim + lane * 4);
-                    m = mml[kDecWarps * kFuRows * 2 - 2];
-                    l = mml[kDecWarps * kFuRows * 2 - 1];
-                }
-#pragma unroll 2
-                for (int p = warp; p < np; p += kDecWarps) {
-                    const float2 ml = st_ml[p];
-                    const float4 v = *reinterpret_cast<const float4 *>(st_o + (size_t)p * kHeadDim + lane * 4);
-                    const float m_new = fmaxf(m, ml.x);
-                    const float sc = fast_exp2(m - m_new), sp = fast_exp2(ml.x - m_new);
-                    acc.x = acc.x * sc + v.x * sp;
-                    acc.y = acc.y * sc + v.y * sp;
-                    acc.z = acc.z * sc + v.z * sp;
-                    acc.w = acc.w * sc + v.w * sp;
-                    l = l * sc + ml.y * sp;
-                    m = m_new;
-                }
-                *reinterpret_cast<float4 *>(mo + (warp * kFuRows) * kFuRowStride + lane * 4) = acc;
-                if (lane == 0) *reinterpret_cast<float2 *>(mml + (warp * kFuRows) * 2) = make_float2(m, l);
-                __syncthreads();
-                if (warp == 0) {
-                    float mm, ll;
-                    const float4 s4 = fu_merge_row(mo, mml, 0, lane, mm, ll);
-                    if (p0 + np < n_part) {          // more rounds to come: keep the state at the end of the buffers
-                        *reinterpret_cast<float4 *>(mo + (size_t)kDecWarps * kFuRows * kFuRowStride - kHeadDim + lane * 4) = s4;
-                        if (lane == 0) {
-                            mml[kDecWarps * kFuRows * 2 - 2] = mm;
-                            mml[kDecWarps * kFuRows * 2 - 1] = ll;
-                        }
-                    } else {
-                        const float inv = ll > 0.f ? 1.0f / ll : 0.f;
-                        uint2 pk;
-                        pk.x = pack_bf16(s4.x * inv, s4.y * inv);
-                        pk.y = pack_bf16(s4.z * inv, s4.w * inv);
-                        *reinterpret_cast<uint2 *>(a.out + ((size_t)db * a.Hq + (size_t)dh * a.G + r) * kHeadDim + lane * 4) = pk;
-                    }
-                }
-                __syncthreads();
-            }
-        }
-        const int helpers = n_part < a.G ? n_part : a.G;
-        if (tid == 0 && s_order == (unsigned)(helpers - 1)) {   // ready for the next launch (stream order)
-            a.tickets[seg] = 0u;
-            a.done[seg] = 0u;
-        }
+        if (!help(s_duty[d][0], c_first, n_part, s_duty[d][3], s_duty[d][4], idx, n_part, n_part < a.G ? n_part : a.G)) return;
     }
 }
 
