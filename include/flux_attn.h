@@ -343,8 +343,8 @@ int flux_plan_set_launch_overlap(flux_plan *plan, int32_t on);
 
 /* Which kernels flux_attn_decode / flux_attn_decode_step launch.  FLUX_DECODE_AUTO (the default)
  * runs the single-launch kernel for batches of at most 32 requests and at most 64 KV heads (one launch
- * does the split-K attention and the merge: the CTA that finishes a (request, KV head) last merges its
- * partials; it covers the batch-1 latency setting of Appendix C.3 and the batched workloads alike) and
+ * does the split-K attention and the merge: the first CTAs of a (request, KV head) merge one query head
+ * each once all its CTAs have announced their partials; it covers the batch-1 latency setting of Appendix C.3 and the batched workloads alike) and
  * the two-launch pair (split-K kernel + combine pass) beyond that; the other two values force one of
  * them where the shape allows.  Both compute Eq. 1 / Eq. 2 over the same rows.  The single-launch
  * kernel is issued with programmatic stream serialisation: it starts with a grid-dependency wait (see
