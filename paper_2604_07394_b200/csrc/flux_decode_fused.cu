@@ -1,8 +1,9 @@
-// Single-launch split-K decode for small batches (sm_100a).
+// Single-launch split-K decode (sm_100a), the default for batches of up to 32 requests.
 //
 // At batch 1 (the latency protocol of Appendix C.3) a sparse layer reads a few megabytes: the
 // launch is bound by fixed costs, not by bandwidth, and a second launch that merges the split-K
-// partials costs as much as the attention itself.  This kernel does the whole layer in one launch:
+// partials costs as much as the attention itself; on the batched workloads the second launch and its
+// partial traffic still cost several per cent.  This kernel does the whole layer in one launch:
 //
 //  * work is split by (request, KV head, 128-token tile): a CTA streams one KV head's 256-byte
 //    row pieces, its eight warps taking 16 tokens each, so a CTA produces partials for the G query
@@ -38,6 +39,8 @@ constexpr int kFuStageBytes = kDecWarps * kDecStages * kDecStageBytes;
 constexpr int kFuMergeOBytes = kDecWarps * kFuRows * kFuRowStride * (int)sizeof(float);
 constexpr int kFuMergeMlBytes = kDecWarps * kFuRows * 2 * (int)sizeof(float);
 constexpr int kFuSmemBytes = kFuStageBytes + kFuMergeOBytes + kFuMergeMlBytes;
+// the kernel's static shared memory (per-request tables for kDecFusedMaxBatch requests) takes the rest of the 227 KB
+static_assert(kFuSmemBytes + 48 * kDecFusedMaxBatch <= 232448, "shared memory per CTA");
 // partial rows (512 bytes of O and 8 bytes of (m, l) each) the idle stage memory takes for the last CTA's merge
 constexpr int kFuStagedRows = kFuStageBytes / (kHeadDim * 4 + 8);
 constexpr long long kFuWaitCycles = 2000000000ll;   // bound of the wait for a segment's arrivals (about a second)
