@@ -349,7 +349,12 @@ int flux_plan_set_launch_overlap(flux_plan *plan, int32_t on);
  * them where the shape allows.  Both compute Eq. 1 / Eq. 2 over the same rows.  The single-launch
  * kernel is issued with programmatic stream serialisation: it starts with a grid-dependency wait (see
  * flux_plan_set_launch_overlap), so results never depend on it, and it lets the next such launch in
- * the stream be set up while it drains. */
+ * the stream be set up while it drains.  Its CTAs (one per SM) wait for one another when they merge
+ * (bounded: about a second), so it expects to get the GPU's SMs while it runs; if other work -- another
+ * stream's long kernel, a second launch of this kernel running at the same time -- keeps some of its
+ * CTAs from starting for that long, the wait expires, FLUX_STATUS_WAIT_EXPIRED is raised and the
+ * outputs of that launch are not valid.  Callers that run several decode streams on one GPU at once
+ * select FLUX_DECODE_TWO_LAUNCH, whose kernels never wait for each other. */
 #define FLUX_DECODE_AUTO          0
 #define FLUX_DECODE_TWO_LAUNCH    1
 #define FLUX_DECODE_SINGLE_LAUNCH 2
