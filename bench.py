@@ -900,11 +900,16 @@ def main():
         sampler2 = ClockSampler(local)
         if rank == 0:
             sampler2.start()
-        sus_ms, sus_steps, sus_bytes, wall0 = 0.0, 0, 0, time.perf_counter()
-        while sus_steps < sus_cap and (time.perf_counter() - wall0) < args.sustain_seconds:
+        # the same number of steps on every rank: from the slowest rank's time for the K steps above
+        step_ms = max_over_ranks(dist, [ms], dev)[0] / K_
+        sus_target = min(sus_cap, (int(args.sustain_seconds * 1e3 / step_ms) // sus_chunk + 1) * sus_chunk)
+        sus_ms, sus_steps, sus_bytes = 0.0, 0, 0
+        barrier()
+        while sus_steps < sus_target:
             sus_ms += timed_replays(db, sus_chunk)
             sus_bytes += sum(db.bytes_step(s_) for s_ in range(t, t + sus_chunk))
             t += sus_chunk; sus_steps += sus_chunk
+        barrier()
         clocks2 = sampler2.stop() if rank == 0 else None
         sus_ms = max_over_ranks(dist, [sus_ms], dev)[0]
         gbs = sus_bytes / (sus_ms * 1e-3) / 1e9
