@@ -731,12 +731,14 @@ def workload_config(w, mask, ctx0):
 
 # ---- small cases for ncu captures ---------------------------------------------------------------
 
-def profile_case(flux, dev, which):
+def profile_case(flux, dev, which, decode_kernel=0):
     """A few launches of one kernel on a case of a few GB whose inputs exceed L2."""
     import dataclasses
     if which == "decode":      # the decode workload cut to 2 layers: same per-launch work as the bench
         w = dataclasses.replace(synth.WORKLOADS["cfg3"], n_layers=2)
         db = DecodeBench(flux, w, dev, 4)
+        db.plan.flux_debug_decode_kernel(decode_kernel)
+        db.plan.flux_plan_set_launch_overlap(True)
         for t in range(2):
             db.step(t)
         torch.cuda.synchronize()
@@ -841,7 +843,8 @@ def main():
     flux.load()
     peaks = measured_peaks()
     if args.profile:
-        profile_case(flux, dev, args.profile)
+        profile_case(flux, dev, args.profile, {"auto": flux.FLUX_DECODE_AUTO, "two_launch": flux.FLUX_DECODE_TWO_LAUNCH,
+                                               "single_launch": flux.FLUX_DECODE_SINGLE_LAUNCH}[args.decode_kernel])
         return
     w = synth.WORKLOADS[args.workload]
     W_, K_ = max(3, args.warmup), args.steps

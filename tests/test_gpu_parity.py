@@ -538,3 +538,71 @@ def test_context_exactly_at_and_beyond_max_context(flux):
     out = plan.flux_attn_prefill(0, 0, qp, k, v, cap - 4)      # the last four positions: fits exactly
     ref = oracle.prefill(oracle.FA, bits(qp), bits(k), bits(v), cap - 4, S, W, _scale())
     compare(out, ref, "prefill chunk ending at max_context")
+
+
+@pytest.mark.parametrize("layout", [0, 1])
+def test_decode_steps_replayed_as_a_graph_stay_correct(flux, layout):
+    """A four-layer decode step (append + attend per layer, single-launch kernel, launch overlap on) captured
+    once as a CUDA graph that also advances its own length vector, replayed 40 times: arrival counters,
+    partial slots and ring slots are reused by every launch, so the last step is checked against the oracle
+    in full, and the caches against the rows every step appended."""
+    Hq, Hkv, S, W, L, T = 8, 2, 16, 48, 4, 40
+    lens0 = [300, 40, 0]                                     # the last request stays inactive
+    B = len(lens0)
+    mask = np.array([[1, 0, 1, 0], [0, 0, 1, 1], [1, 1, 0, 0]], dtype=np.uint8)
+    cap = max(lens0) + T + 2
+    plan = _plan(flux, L, Hq, Hkv, S, W, B, cap, layout, 3)
+    plan.flux_router_apply(mask=mask)
+    kc, vc, klog, vlog = [], [], [], []
+    for layer in range(L):
+        kl, vl, kg, vg = [], [], [], []
+        for b, n in enumerate(lens0):
+            compact = layout == 1 and mask[b, layer] == 0
+            k = synth.normal_bf16((cap, Hkv, 128), 61, 10 * layer + b, DEV)
+            v = synth.normal_bf16((cap, Hkv, 128), 62, 10 * layer + b, DEV)
+            kcache = torch.zeros((S + W if compact else cap, Hkv, 128), dtype=torch.bfloat16, device=DEV)
+            vcache = torch.zeros_like(kcache)
+            if n > 0:
+                plan.flux_kv_retain(layer, b, k, v, n, kcache, vcache)
+            kl.append(kcache); vl.append(vcache); kg.append(k.cpu().clone()); vg.append(v.cpu().clone())
+        kc.append(kl); vc.append(vl); klog.append(kg); vlog.append(vg)
+    ktab = [flux.pointer_table(kc[l], DEV) for l in range(L)]
+    vtab = [flux.pointer_table(vc[l], DEV) for l in range(L)]
+    q = synth.normal_bf16((L, B, Hq, 128), 63, 0, DEV)
+    kn = synth.normal_bf16((L, B, Hkv, 128), 64, 0, DEV)      # the same new rows every step: what matters is where they land
+    vn = synth.normal_bf16((L, B, Hkv, 128), 65, 0, DEV)
+    out = torch.zeros_like(q)
+    active = torch.tensor([1 if n > 0 else 0 for n in lens0], dtype=torch.int32, device=DEV)
+    ctx = torch.tensor([n + 1 if n > 0 else 0 for n in lens0], dtype=torch.int32, device=DEV)   # length incl. the new token
+
+    def step():
+        for l in range(L):
+            plan.flux_attn_decode_step(l, B, q[l], kn[l], vn[l], ktab[l], vtab[l], ctx, out[l])
+
+    step()                                                   # eager once (also loads everything the capture must not)
+    ctx += active
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+        ctx += active
+    for _ in range(T - 2):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert plan.flux_plan_status() == 0
+    # one eager step and T - 2 replays have run (capturing only records)
+    steps_done = 1 + (T - 2)
+    for b, n0 in enumerate(lens0):
+        if n0 == 0:
+            assert torch.count_nonzero(out[:, b]) == 0
+            continue
+        n = n0 + steps_done                                  # context length seen by the last step
+        for l in range(L):
+            mode = int(mask[b, l])
+            kfull, vfull = klog[l][b].clone(), vlog[l][b].clone()
+            kfull[n0:n] = kn[l, b].cpu(); vfull[n0:n] = vn[l, b].cpu()
+            ref = oracle.decode(mode, bits(q[l, b]), bits(kfull), bits(vfull), n, S, W, _scale())
+            compare(out[l, b], ref, "graph replay b=%d layer=%d mode=%d" % (b, l, mode))
+            compact = layout == 1 and mode == 0
+            keep = oracle.retained(n, S, W) if mode == 0 else np.arange(n)
+            assert torch.equal(logical_view(kc[l][b], n, S, W, compact)[keep], kfull[:n][keep])
