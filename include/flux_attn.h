@@ -103,9 +103,15 @@ int flux_plan_set_workspace(flux_plan *plan, void *workspace /*device*/, size_t 
  *                    w_enc1 [E][2*Hq*D], w_enc2 [E][E], w_head1 [R][E], w_head2 [2][R] (row 0 = FA).
  *   logits_out       fp32 [2] on the device, 8-byte aligned, e.g. the (request, layer) slot of the
  *                    [B][n_layers][2] array later given to flux_router_apply.
- * Five launches on `stream` (pooling + four matrix-vector products, fp32 accumulation); scratch is
- * in the workspace, so calls for different layers must be stream-ordered.  Cost does not depend
- * on the prompt length.  Errors: NULL / misaligned pointers, n_* < 1 -> FLUX_E_INVALID_ARG; widths
+ * One launch on `stream` (pooling + four matrix-vector products, fp32 accumulation, a fixed
+ * summation order); scratch is in the workspace, so calls for different layers must be
+ * stream-ordered.  Cost does not depend on the prompt length.  The launch may begin while the
+ * kernel before it in the stream is still draining, and reads the WEIGHTS AND BIASES (nothing
+ * else) before that kernel has finished: the work enqueued immediately before this call must not
+ * be what writes them.  The kernel's CTAs (one per SM) wait for one another between stages; the
+ * waits are bounded (about a second, then FLUX_STATUS_WAIT_EXPIRED in the status word and
+ * unspecified logits), which only a kernel of another stream that holds SMs for that long can
+ * cause.  Errors: NULL / misaligned pointers, n_* < 1 -> FLUX_E_INVALID_ARG; widths
  * not multiples of 8 -> FLUX_E_UNSUPPORTED_SHAPE; widths > 4096 -> FLUX_E_CAPACITY. */
 typedef struct {
     int32_t enc_dim;       /* E */
