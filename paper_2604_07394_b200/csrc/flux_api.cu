@@ -104,8 +104,8 @@ WorkspaceLayout workspace_layout(const flux_config &c)
     w.host_k = off;       off = align_up(off + B * c.n_kv_heads * kRowBytes, A);
     w.host_v = off;       off = align_up(off + B * c.n_kv_heads * kRowBytes, A);
     w.host_o = off;       off = align_up(off + B * c.n_q_heads * kRowBytes, A);
-    w.router = off;       off = align_up(off + ((size_t)2 * c.n_q_heads * kHeadDim + 3 * kRouterMaxWidth) * sizeof(float), A);
-    w.router_sync = off;  off = align_up(off + 4 * sizeof(uint32_t), A);
+    w.router = off;       off = align_up(off + ((size_t)2 * c.n_q_heads * kHeadDim + 6 * kRouterMaxWidth) * sizeof(float), A);
+    w.router_sync = off;  off = align_up(off + 8 * sizeof(uint32_t), A);
     w.tickets = off;      off = align_up(off + 2 * (size_t)kDecFusedMaxBatch * c.n_kv_heads * sizeof(uint32_t), A);
     w.total = off;
     return w;
@@ -772,7 +772,9 @@ int flux_plan_status(flux_plan *plan, uint32_t *status_bits, void *stream)
     if (!rc) rc = check_cuda(cudaStreamSynchronize(st), "stream synchronize");
     if (rc) return rc;
     if (bits & FLUX_STATUS_WAIT_EXPIRED) {   // a kernel left early: its arrival counters are not back at zero
-        rc = check_cuda(cudaMemsetAsync((char *)plan->ws + plan->lay.router_sync, 0, 4 * sizeof(uint32_t), st), "counter clear");
+        // the router's counters and launch number, and with them the tagged activations (an old tag must not match)
+        rc = check_cuda(cudaMemsetAsync((char *)plan->ws + plan->lay.router, 0,
+                                        plan->lay.router_sync + 8 * sizeof(uint32_t) - plan->lay.router, st), "counter clear");
         if (!rc) rc = check_cuda(cudaMemsetAsync((char *)plan->ws + plan->lay.tickets, 0,
                                                  2 * (size_t)kDecFusedMaxBatch * plan->cfg.n_kv_heads * sizeof(uint32_t), st), "counter clear");
         if (!rc) rc = check_cuda(cudaStreamSynchronize(st), "stream synchronize");

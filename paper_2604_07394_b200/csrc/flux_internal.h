@@ -38,8 +38,8 @@ struct WorkspaceLayout {
     size_t host_k;       // bf16  [max_batch][Hkv][D]
     size_t host_v;       // bf16  [max_batch][Hkv][D]
     size_t host_o;       // bf16  [max_batch][Hq][D]
-    size_t router;       // fp32  [2*Hq*D + 3*kRouterMaxWidth] pooled descriptor and hidden activations
-    size_t router_sync;  // uint32 [4] barrier counters and ticket of the one-launch router front end (zero between launches)
+    size_t router;       // fp32 [2*Hq*D] pooled descriptor, then uint64 [3][kRouterMaxWidth] hidden activations (value | launch number << 32)
+    size_t router_sync;  // uint32 [8]: barrier counter and exit ticket of the router front end (zero between launches), its launch number
     size_t tickets;      // uint32 [2][kDecFusedMaxBatch][Hkv] arrival / helper counters of the single-launch decode (zero between launches)
     size_t total;
     int64_t slots;

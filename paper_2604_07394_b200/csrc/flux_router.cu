@@ -6,13 +6,15 @@
 //
 // The work is tiny and independent of the prompt length (at most 200 tokens of x_Q, a few MB of
 // weights), so it is bound by launch and dependency latency, not by bandwidth.  One launch of one
-// CTA per SM runs all five stages -- pooling, the four matrix-vector products -- with a grid-wide
-// barrier (bounded spin on an arrival counter; a grid of one CTA per SM, each taking a whole SM's
-// shared memory, is resident as soon as the kernel before it has left) between a stage and the
-// next one that needs its whole output; the last stage, two rows, is done by the CTA that
-// finishes the one before it last.  The launch allows programmatic overlap with the kernel before
-// it in the stream: the weight rows are requested while that kernel drains.  fp32 accumulation,
-// bf16 weights, deterministic reduction order.
+// CTA per SM runs all five stages -- pooling, the four matrix-vector products.  The pooled
+// descriptor is handed to the first product through a grid-wide barrier (bounded spin on an
+// arrival counter; a grid of one CTA per SM is resident as soon as the kernel before it has
+// left).  The later activations are small, so each value travels with a tag -- the launch's
+// number -- in one 64-bit word, and a consumer simply re-reads its inputs until their tags are
+// this launch's: one trip to L2 after the producer's store instead of a barrier plus a read.
+// The launch allows programmatic overlap with the kernel before it in the stream: the weight
+// rows are requested while that kernel drains.  fp32 accumulation, bf16 weights, deterministic
+// reduction order.
 #include "flux_internal.h"
 #include "flux_mma_util.h"
 #include "flux_tc_util.h"
@@ -31,8 +33,9 @@ struct RouterArgs {
     const __nv_bfloat16 *w1, *w2, *w3, *w4;
     const float *b1, *b2, *b3, *b4;
     int F, E, R;
-    float *f, *h1, *u, *h2, *logits;
-    unsigned *sync;                      // [4]: three barrier counters, one ticket; zero between launches
+    float *f, *logits;
+    unsigned long long *h1, *u, *h2;     // tagged activations: low word the fp32 value, high word the launch number
+    unsigned *sync;                      // [0] barrier counter, [1] exit ticket (both zero between launches), [2] last launch number
     uint32_t *status;
     int pre_bytes, pre_off[3];           // shared memory: eight areas of pre_bytes, one per output row of a CTA's first pass;
                                          // byte offset of the row of stage 1 / 2 / 3 in an area, -1: not brought in ahead
@@ -74,8 +77,33 @@ constexpr int kRouterWarps = 16;
 // weights and the input vector are each read once per CTA.  fp32 FMAs in a fixed order; per row a butterfly over the
 // lanes, then the sixteen warps' sums added in warp order.  `pre`: the CTA's first eight rows (row r at
 // pre + r * pre_stride), brought into shared memory by the bulk copies issued at the start of the kernel, or NULL.
-// `bias0`: b[row] of the first pass for threads 0..7, read at the start of the kernel (a late read would put one more
-// trip to memory on the critical path).
+__device__ __forceinline__ void st_tagged(unsigned long long *p, float v, unsigned epoch)
+{
+    const unsigned long long w = ((unsigned long long)epoch << 32) | (unsigned long long)__float_as_uint(v);
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;\n" ::"l"(p), "l"(w) : "memory");
+}
+
+// The eight tagged inputs of piece i, re-read until every tag is this launch's.  false: the wait ran out.
+__device__ __forceinline__ bool ld_tagged_piece(const unsigned long long *x, int i, unsigned epoch, float4 &x0, float4 &x1)
+{
+    unsigned long long w[8];
+    long long t0 = 0;
+    for (;;) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];\n" : "=l"(w[2 * k]), "=l"(w[2 * k + 1]) : "l"(x + 8 * (size_t)i + 2 * k) : "memory");
+        bool ok = true;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) ok = ok && (unsigned)(w[k] >> 32) == epoch;
+        if (ok) break;
+        if (t0 == 0) t0 = clock64();
+        else if (clock64() - t0 > kRouterWaitCycles) return false;
+    }
+    x0 = make_float4(__uint_as_float((unsigned)w[0]), __uint_as_float((unsigned)w[1]), __uint_as_float((unsigned)w[2]), __uint_as_float((unsigned)w[3]));
+    x1 = make_float4(__uint_as_float((unsigned)w[4]), __uint_as_float((unsigned)w[5]), __uint_as_float((unsigned)w[6]), __uint_as_float((unsigned)w[7]));
+    return true;
+}
+
 __device__ __forceinline__ void accumulate_piece(float (&acc)[8][2], const uint4 p, const float4 x0, const float4 x1, int r)
 {
     const float2 w0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&p.x));
@@ -86,29 +114,37 @@ __device__ __forceinline__ void accumulate_piece(float (&acc)[8][2], const uint4
     acc[r][1] = fmaf(w3.y, x1.w, fmaf(w3.x, x1.z, fmaf(w2.y, x1.y, fmaf(w2.x, x1.x, acc[r][1]))));
 }
 
-__device__ __forceinline__ void linear_stage(const __nv_bfloat16 *__restrict__ W, const float *__restrict__ b, const float *x,
-                                             float *y, int n_in, int n_out, int act, const unsigned char *pre,
-                                             size_t pre_stride, float bias0, float (*s_part)[8])
+// x_plain: the input as plain floats (complete: a grid-wide barrier came before); else x_tagged.  The output is
+// tagged.  `bias0`: b[row] of the first pass for threads 0..7, read at the start of the kernel (a late read would put
+// one more trip to memory on the critical path).  false: a wait ran out (flagged), the caller leaves.
+__device__ __forceinline__ bool linear_stage(const __nv_bfloat16 *__restrict__ W, const float *__restrict__ b, const float *x_plain,
+                                             const unsigned long long *x_tagged, unsigned long long *y, int n_in, int n_out,
+                                             int act, const unsigned char *pre, size_t pre_stride, float bias0, unsigned epoch,
+                                             float (*s_part)[8], int *s_abort, uint32_t *status)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int n_pieces = n_in / 8;
     const int base0 = (int)blockIdx.x * 8;
     for (int base = base0; base < n_out; base += (int)gridDim.x * 8) {
+        const bool staged = pre != nullptr && base == base0;   // rows in shared memory (rows beyond n_out were not copied and are skipped)
         float acc[8][2];
 #pragma unroll
         for (int r = 0; r < 8; ++r) acc[r][0] = acc[r][1] = 0.f;
-        if (pre != nullptr && base == base0) {          // rows in shared memory (rows beyond n_out were not copied and are skipped)
-            for (int i = warp * 32 + lane; i < n_pieces; i += kRouterWarps * 32) {
-                const float4 x0 = __ldcg(reinterpret_cast<const float4 *>(x) + 2 * i);
-                const float4 x1 = __ldcg(reinterpret_cast<const float4 *>(x) + 2 * i + 1);
+        for (int i = warp * 32 + lane; i < n_pieces; i += kRouterWarps * 32) {
+            float4 x0, x1;
+            if (x_plain) {
+                x0 = __ldcg(reinterpret_cast<const float4 *>(x_plain) + 2 * i);
+                x1 = __ldcg(reinterpret_cast<const float4 *>(x_plain) + 2 * i + 1);
+            } else if (!ld_tagged_piece(x_tagged, i, epoch, x0, x1)) {
+                atomicOr(status, FLUX_STATUS_WAIT_EXPIRED);
+                *reinterpret_cast<volatile int *>(s_abort) = 1;
+                break;
+            }
+            if (staged) {
 #pragma unroll
                 for (int r = 0; r < 8; ++r)
                     if (base + r < n_out) accumulate_piece(acc, reinterpret_cast<const uint4 *>(pre + r * pre_stride)[i], x0, x1, r);
-            }
-        } else {
-            for (int i = warp * 32 + lane; i < n_pieces; i += kRouterWarps * 32) {
-                const float4 x0 = __ldcg(reinterpret_cast<const float4 *>(x) + 2 * i);
-                const float4 x1 = __ldcg(reinterpret_cast<const float4 *>(x) + 2 * i + 1);
+            } else {
 #pragma unroll
                 for (int r = 0; r < 8; ++r)
                     if (base + r < n_out)
@@ -123,15 +159,17 @@ __device__ __forceinline__ void linear_stage(const __nv_bfloat16 *__restrict__ W
             if (lane == 0) s_part[warp][r] = v;
         }
         __syncthreads();
+        if (*reinterpret_cast<volatile int *>(s_abort)) return false;
         if (threadIdx.x < 8 && base + (int)threadIdx.x < n_out) {
             float v = s_part[0][threadIdx.x];
 #pragma unroll
             for (int w = 1; w < kRouterWarps; ++w) v += s_part[w][threadIdx.x];
             v += base == base0 ? bias0 : b[base + threadIdx.x];
-            y[base + threadIdx.x] = act ? silu(v) : v;
+            st_tagged(y + base + threadIdx.x, act ? silu(v) : v, epoch);
         }
         __syncthreads();
     }
+    return true;
 }
 
 constexpr int kRouterThreads = kRouterWarps * 32;
@@ -143,7 +181,6 @@ __global__ void __launch_bounds__(kRouterThreads) router_fused_kernel(RouterArgs
     __shared__ float2 part[16][32];
     __shared__ float s_part[kRouterWarps][8];
     __shared__ int s_abort;
-    __shared__ unsigned s_ticket;
     __shared__ __align__(8) unsigned long long s_bar[3];   // weight rows of stage 1 / 2 / 3 have landed
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // The launch is issued with programmatic stream serialisation: dependents are released at once, and the weights
@@ -178,8 +215,8 @@ __global__ void __launch_bounds__(kRouterThreads) router_fused_kernel(RouterArgs
             }
         }
     }
-    // constants that sit on the critical path later: the biases of this CTA's first rows, and (in every CTA, since
-    // the one that will finish last is not known) the two rows of the last stage
+    // constants that sit on the critical path later: the biases of this CTA's first rows and, in the last CTA (which
+    // has the fewest rows and computes the logits), the two rows of the last stage
     float bias0[3] = {0.f, 0.f, 0.f};
     if (tid < 8) {
         const int row0 = (int)blockIdx.x * 8 + tid;
@@ -188,7 +225,8 @@ __global__ void __launch_bounds__(kRouterThreads) router_fused_kernel(RouterArgs
     }
     uint4 w4_early[kRouterLastEarly];
     float b4_early = 0.f;
-    if (warp < 2) {
+    const bool does_logits = blockIdx.x == gridDim.x - 1;
+    if (does_logits && warp < 2) {
 #pragma unroll
         for (int j = 0; j < kRouterLastEarly; ++j) {
             const int i = lane + 32 * j;
@@ -197,7 +235,9 @@ __global__ void __launch_bounds__(kRouterThreads) router_fused_kernel(RouterArgs
         b4_early = __ldg(a.b4 + warp);
     }
     asm volatile("griddepcontrol.wait;\n" ::: "memory");
-    // ---- pooling: a CTA takes 32 bf16x2 columns of one segment at a time; warp w sums tokens w, w + 16, ... ----
+    unsigned epoch = __ldcg(a.sync + 2) + 1u;      // this launch's number (the one before it has finished and stored its own)
+    if (epoch == 0u) epoch = 1u;                    // zero is what a cleared buffer holds
+    // ---- pooling: a CTA takes 32 bf16x2 columns of one segment at a time; warp w sums tokens w, w + 16, ... (in that order) ----
     const int slabs = (a.F2 + 31) / 32;
     for (int item = blockIdx.x; item < 2 * slabs; item += gridDim.x) {
         const int seg = item / slabs, col = (item % slabs) * 32 + lane;
@@ -205,11 +245,20 @@ __global__ void __launch_bounds__(kRouterThreads) router_fused_kernel(RouterArgs
         const int n = seg ? a.n_last : a.n_first;
         float2 acc = make_float2(0.f, 0.f);
         if (col < a.F2) {
-#pragma unroll 8
-            for (int t = warp; t < n; t += 16) {
-                const float2 v = __bfloat1622float2(x[(size_t)t * a.F2 + col]);
-                acc.x += v.x;
-                acc.y += v.y;
+            // eight loads in flight per lane (a loop with a data-dependent trip count would take them one by one)
+            for (int t0 = warp; t0 < n; t0 += 8 * kRouterWarps) {
+                __nv_bfloat162 v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const int t = t0 + j * kRouterWarps;
+                    v[j] = t < n ? x[(size_t)t * a.F2 + col] : __float2bfloat162_rn(0.f);
+                }
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const float2 f2 = __bfloat1622float2(v[j]);
+                    acc.x += f2.x;
+                    acc.y += f2.y;
+                }
             }
         }
         __syncthreads();      // the previous item's sums have been read
@@ -240,28 +289,22 @@ __global__ void __launch_bounds__(kRouterThreads) router_fused_kernel(RouterArgs
     auto leave = [&]() { for (int s = 0; s < 3; ++s) rows_landed(s); };
     if (!grid_barrier(a.sync + 0, a.status, &s_abort)) { leave(); return; }
     if (!rows_landed(0)) { leave(); return; }
-    linear_stage(a.w1, a.b1, a.f, a.h1, a.F, a.E, 1, a.pre_off[0] >= 0 ? rows + a.pre_off[0] : nullptr, (size_t)a.pre_bytes, bias0[0], s_part);
-    if (!grid_barrier(a.sync + 1, a.status, &s_abort)) { leave(); return; }
+    if (!linear_stage(a.w1, a.b1, a.f, nullptr, a.h1, a.F, a.E, 1, a.pre_off[0] >= 0 ? rows + a.pre_off[0] : nullptr,
+                      (size_t)a.pre_bytes, bias0[0], epoch, s_part, &s_abort, a.status)) { leave(); return; }
     if (!rows_landed(1)) { leave(); return; }
-    linear_stage(a.w2, a.b2, a.h1, a.u, a.E, a.E, 0, a.pre_off[1] >= 0 ? rows + a.pre_off[1] : nullptr, (size_t)a.pre_bytes, bias0[1], s_part);
-    if (!grid_barrier(a.sync + 2, a.status, &s_abort)) { leave(); return; }
+    if (!linear_stage(a.w2, a.b2, nullptr, a.h1, a.u, a.E, a.E, 0, a.pre_off[1] >= 0 ? rows + a.pre_off[1] : nullptr,
+                      (size_t)a.pre_bytes, bias0[1], epoch, s_part, &s_abort, a.status)) { leave(); return; }
     if (!rows_landed(2)) { leave(); return; }
-    linear_stage(a.w3, a.b3, a.u, a.h2, a.E, a.R, 1, a.pre_off[2] >= 0 ? rows + a.pre_off[2] : nullptr, (size_t)a.pre_bytes, bias0[2], s_part);
-    // ---- the two logits: by the CTA that finishes the stage above last ----
-    __syncthreads();
-    if (tid == 0) {
-        unsigned ticket;
-        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;\n" : "=r"(ticket) : "l"(a.sync + 3) : "memory");
-        s_ticket = ticket;
-    }
-    __syncthreads();
-    if (s_ticket != gridDim.x - 1) return;
-    if (warp < 2) {
+    if (!linear_stage(a.w3, a.b3, nullptr, a.u, a.h2, a.E, a.R, 1, a.pre_off[2] >= 0 ? rows + a.pre_off[2] : nullptr,
+                      (size_t)a.pre_bytes, bias0[2], epoch, s_part, &s_abort, a.status)) { leave(); return; }
+    // ---- the two logits ----
+    if (does_logits && warp < 2) {
         const uint4 *w = reinterpret_cast<const uint4 *>(a.w4 + (size_t)warp * a.R);
-        const float4 *xv = reinterpret_cast<const float4 *>(a.h2);
         float acc = 0.f;
+        bool ok = true;
         auto piece = [&](const uint4 p, int i) {
-            const float4 x0 = __ldcg(xv + 2 * i), x1 = __ldcg(xv + 2 * i + 1);
+            float4 x0, x1;
+            if (!ld_tagged_piece(a.h2, i, epoch, x0, x1)) { ok = false; return; }
             const float2 w0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&p.x));
             const float2 w1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&p.y));
             const float2 w2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&p.z));
@@ -278,12 +321,26 @@ __global__ void __launch_bounds__(kRouterThreads) router_fused_kernel(RouterArgs
 #pragma unroll
         for (int j = 0; j < kRouterLastEarly; ++j)
             if (lane + 32 * j < a.R / 8) piece(w4_early[j], lane + 32 * j);
-        for (int i = lane + 32 * kRouterLastEarly; i < a.R / 8; i += 32) piece(__ldg(w + i), i);
+        for (int i = lane + 32 * kRouterLastEarly; i < a.R / 8 && ok; i += 32) piece(__ldg(w + i), i);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        if (lane == 0) a.logits[warp] = acc + b4_early;
+        if (!__all_sync(0xffffffffu, ok)) {
+            if (lane == 0) atomicOr(a.status, FLUX_STATUS_WAIT_EXPIRED);
+        } else if (lane == 0) {
+            a.logits[warp] = acc + b4_early;
+        }
     }
-    if (tid < 4) a.sync[tid] = 0u;   // ready for the next launch (every other CTA is past all of them)
+    // ---- the CTA that leaves last puts the counters back and records the launch number ----
+    __syncthreads();
+    if (tid == 0) {
+        unsigned ticket;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;\n" : "=r"(ticket) : "l"(a.sync + 1) : "memory");
+        if (ticket == gridDim.x - 1) {
+            a.sync[0] = 0u;
+            a.sync[1] = 0u;
+            a.sync[2] = epoch;
+        }
+    }
 }
 
 constexpr int kRouterSmemLimit = 227 * 1024 - 5120;   // dynamic shared memory the kernel may ask for (its static part is about 4.6 KB)
@@ -301,7 +358,8 @@ int launch_router_frontend(flux_plan *p, const flux_router_weights *w, const voi
 {
     const int F1 = p->cfg.n_q_heads * kHeadDim, F = 2 * F1, E = w->enc_dim, R = w->head_hidden;
     float *scr = (float *)((char *)p->ws + p->lay.router);
-    float *f = scr, *h1 = f + F, *u = h1 + kRouterMaxWidth, *h2 = u + kRouterMaxWidth;
+    float *f = scr;
+    unsigned long long *h1 = reinterpret_cast<unsigned long long *>(f + F), *u = h1 + kRouterMaxWidth, *h2 = u + kRouterMaxWidth;
     {
         RouterArgs a;
         a.first = (const __nv_bfloat162 *)q_first; a.last = (const __nv_bfloat162 *)q_last;
