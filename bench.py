@@ -399,7 +399,7 @@ def router_frontend_block(flux, dev, peaks, warmup, enc_dim=1024, head_hidden=25
             "us_per_layer_call_by_call": ms_eager * 1e3 / L,
             "algorithmic_bytes_per_layer": bytes_layer,
             "gbs": bytes_layer * L / (ms * 1e-3) / 1e9, "hbm_peak_gbs": peaks["hbm_gbs"],
-            "bound": "dependency latency (%d launch per layer with three grid-wide barriers, %.1f MB of weights per layer)"
+            "bound": "dependency latency (%d launch per layer, five dependent stages handed over through L2, %.1f MB of weights per layer)"
                      % ((launches - 1) // L, bytes_layer / 1e6),
             "hbm_floor_us_per_layer": bytes_layer / (peaks["hbm_gbs"] * 1e9) * 1e6,
             "gpu_launches": launches,
