@@ -772,6 +772,20 @@ def profile_case(flux, dev, which, decode_kernel=0):
         i = np.arange(N, dtype=np.int64)
         print(json.dumps({"profile_case": "prefill32k", "N": N, "launches": 2, "device_gb": 4 * q.numel() * 2 / 1e9 * 0.625,
                           "flop_per_launch": 4 * w.n_q_heads * D * int((i + 1).sum())}))
+    elif which == "router":    # the router front end of the benchmark's stack: 16 layers of weights (beyond L2), two passes
+        w = synth.WORKLOADS["cfg2"]
+        L, Hq = 16, w.n_q_heads
+        plan = flux.Plan(flux.make_config(L, Hq, w.n_kv_heads, w.sink, w.window, 1, 4096), dev)
+        q = synth.normal_bf16((4096, Hq, D), w.seed, synth.stream_id("q"), dev)
+        ws = [synth.router_weights(w.seed, l, 2 * Hq * D, 1024, 256, dev) for l in range(L)]
+        logits = torch.zeros((1, L, 2), dtype=torch.float32, device=dev)
+        for _ in range(2):
+            for l in range(L):
+                plan.flux_router_forward(ws[l], q[:100], q[-100:], logits[0, l])
+        torch.cuda.synchronize()
+        assert plan.flux_plan_status() == 0
+        print(json.dumps({"profile_case": "router", "layers": L, "launches": 2 * L,
+                          "weight_bytes_per_launch": 2 * (2 * Hq * D * 1024 + 1024 * 1024 + 256 * 1024 + 2 * 256)}))
     elif which == "heads":     # one dense, one sparse and one half-sparse-heads layer call at 256K tokens
         res = head_level_block(flux, dev, measured_peaks(), 1, reps=1)
         print(json.dumps({"profile_case": "heads", "launch_order": "each of dense, sparse, head-level: 3 warm-up + 1",
@@ -815,7 +829,7 @@ def main():
                     help="skip the other decode workloads (cfg4, cfg5) and the 128K prefill layers")
     ap.add_argument("--sustain-seconds", type=float, default=3.0,
                     help="after the K timed steps, keep replaying the step for this long and report the sustained rate")
-    ap.add_argument("--profile", default=None, choices=["decode", "decode_b1", "prefill", "prefill32k", "heads"],
+    ap.add_argument("--profile", default=None, choices=["decode", "decode_b1", "prefill", "prefill32k", "heads", "router"],
                     help="run a small case of one kernel with few launches (for ncu captures) and exit")
     args = ap.parse_args()
     if args.impl == "reference":
