@@ -85,3 +85,63 @@ def test_router_forward_rejects_bad_arguments(flux):
         plan.flux_router_forward(w, q, q, torch.zeros(2, dtype=torch.float32))     # host logits_out
     assert e.value.code == flux.FLUX_E_INVALID_ARG
     assert plan.flux_plan_status() == 0
+
+
+def _router_case(Hq=32, Hkv=8, E=256, R=64, N=600, L=3):
+    q = synth.normal_bf16((N, Hq, 128), 91, synth.stream_id("q"), DEV)
+    ws = [synth.router_weights(91, layer, 2 * Hq * 128, E, R, DEV) for layer in range(L)]
+    first, last = q[:100], q[-100:]
+    ref = np.stack([rf.logits(oracle.to_bits(first.cpu()), oracle.to_bits(last.cpu()), _bits(w)) for w in ws])
+    return ws, first, last, ref
+
+
+def test_router_forward_in_a_replayed_graph(flux):
+    """The kernel tells this launch's activations from an older launch's by a launch number kept on the
+    device: a captured graph replays the same arguments, so every replay must still find fresh values.
+    Logits after each of several replays equal the oracle's; a call issued outside the graph between
+    replays (one more launch number) changes nothing."""
+    ws, first, last, ref = _router_case()
+    plan = flux.Plan(flux.make_config(3, 32, 8, 64, 256, 1, 1024), DEV)
+    logits = torch.zeros((1, 3, 2), dtype=torch.float32, device=DEV)
+
+    def one_pass():
+        for layer, w in enumerate(ws):
+            plan.flux_router_forward(w, first, last, logits[0, layer])
+
+    one_pass()                                      # first use outside capture
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        one_pass()
+    for rep in range(6):
+        logits.fill_(float("nan"))
+        graph.replay()
+        if rep == 3:
+            plan.flux_router_forward(ws[1], first, last, logits[0, 1])
+        torch.cuda.synchronize()
+        got = logits[0].cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - ref) <= 1e-4 * (1.0 + np.abs(ref))), (rep, got, ref)
+    assert plan.flux_plan_status() == 0
+
+
+def test_router_forward_after_a_cleared_timeout(flux):
+    """Reading a status word that reports a timed-out wait puts the router's counters and its launch number
+    back to zero (a kernel that gave up leaves them anywhere); the tagged activations are cleared with them,
+    so the launches that follow start again from launch number one and are correct."""
+    ws, first, last, ref = _router_case(L=2)
+    plan = flux.Plan(flux.make_config(2, 32, 8, 64, 256, 1, 1024), DEV)
+    logits = torch.zeros((1, 2, 2), dtype=torch.float32, device=DEV)
+    for rounds in range(2):
+        for _ in range(3):                          # launch numbers 1..6 leave their tags behind
+            for layer, w in enumerate(ws):
+                plan.flux_router_forward(w, first, last, logits[0, layer])
+        plan.flux_debug_wait_probe(2_000_000)       # a bounded wait that runs out: the status bit, nothing else
+        with pytest.raises(flux.FluxError) as e:
+            plan.flux_plan_status()
+        assert e.value.code == flux.FLUX_E_DEVICE_TIMEOUT
+        logits.fill_(float("nan"))
+        for layer, w in enumerate(ws):
+            plan.flux_router_forward(w, first, last, logits[0, layer])
+        got = logits[0].cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(got - ref) <= 1e-4 * (1.0 + np.abs(ref))), (rounds, got, ref)
+        assert plan.flux_plan_status() == 0
