@@ -482,6 +482,22 @@ def prefill_block(flux, dev, peaks, warmup):
                             "streaming at block granularity: %d sink + %d local blocks" % (-(-S // 64), -(-W // 64)),
                             "ms_layer": ms_blk, "tflops": 4 * Hq * D * pairs_blk / ms_blk / 1e9}
     if ms_fa is not None:
+        # the same FA launch timed alone: one launch after the GPU has been idle for a while, which is how the burst
+        # peak of the roofline's denominator was taken (the loop above runs under the power cap, like the sustained one)
+        alone = []
+        for _ in range(3):
+            time.sleep(1.5)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            plan.flux_attn_prefill(fa_layers[0], 0, q, k, v, 0, out)
+            e1.record()
+            torch.cuda.synchronize()
+            alone.append(e0.elapsed_time(e1))
+        ms_alone = sorted(alone)[1]
+        res["fa_layer_timed_alone"] = {"ms": ms_alone, "tflops": flop_fa / ms_alone / 1e9,
+                                       "frac_of_burst_peak": flop_fa / ms_alone / 1e9 / peaks["bf16_tflops"],
+                                       "how": "one launch after 1.5 s of idle, event-timed, median of 3 (%s ms)"
+                                              % ", ".join("%.3f" % x for x in alone)}
         ach = flop_fa / ms_fa / 1e9
         res["roofline"] = {"bound": "tensor", "achieved": ach, "peak": peaks["bf16_tflops_sustained"],
                            "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops_sustained"],

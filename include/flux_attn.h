@@ -276,7 +276,11 @@ int flux_attn_prefill_host(flux_plan *plan, int32_t layer, int32_t req, const vo
 
 /* Synchronises `stream`, reads the device status word and clears it.  Returns
  * FLUX_OK with *status_bits == 0, FLUX_E_DEVICE_TIMEOUT if a wait expired, or
- * FLUX_E_DEVICE_FLAG for the input-check bits.  status_bits (host) may be NULL. */
+ * FLUX_E_DEVICE_FLAG for the input-check bits.  status_bits (host) may be NULL.
+ * A kernel that gave up on a wait leaves its hand-over state in the workspace wherever it
+ * stood; when the word reports a timeout this call also puts that state (the arrival counters
+ * of the single-launch decode, the router front end's counters, launch number and tagged
+ * activations) back to zero on `stream`, so the calls that follow start clean. */
 int flux_plan_status(flux_plan *plan, uint32_t *status_bits, void *stream);
 
 /* Dispatch record of the latest flux_attn_decode / flux_attn_prefill on this
