@@ -178,7 +178,7 @@ constexpr int kRouterLastEarly = 2;   // 16-byte pieces per lane of a last-stage
 __global__ void __launch_bounds__(kRouterThreads) router_fused_kernel(RouterArgs a)
 {
     extern __shared__ __align__(16) unsigned char rows[];
-    __shared__ float2 part[16][32];
+    __shared__ float2 part[kRouterWarps][32];
     __shared__ float s_part[kRouterWarps][8];
     __shared__ int s_abort;
     __shared__ __align__(8) unsigned long long s_bar[3];   // weight rows of stage 1 / 2 / 3 have landed
@@ -237,7 +237,7 @@ __global__ void __launch_bounds__(kRouterThreads) router_fused_kernel(RouterArgs
     asm volatile("griddepcontrol.wait;\n" ::: "memory");
     unsigned epoch = __ldcg(a.sync + 2) + 1u;      // this launch's number (the one before it has finished and stored its own)
     if (epoch == 0u) epoch = 1u;                    // zero is what a cleared buffer holds
-    // ---- pooling: a CTA takes 32 bf16x2 columns of one segment at a time; warp w sums tokens w, w + 16, ... (in that order) ----
+    // ---- pooling: a CTA takes 32 bf16x2 columns of one segment at a time; warp w sums tokens w, w + kRouterWarps, ... (in that order) ----
     const int slabs = (a.F2 + 31) / 32;
     for (int item = blockIdx.x; item < 2 * slabs; item += gridDim.x) {
         const int seg = item / slabs, col = (item % slabs) * 32 + lane;
@@ -267,7 +267,7 @@ __global__ void __launch_bounds__(kRouterThreads) router_fused_kernel(RouterArgs
         if (warp == 0 && col < a.F2) {
             float2 sum = part[0][lane];
 #pragma unroll
-            for (int g = 1; g < 16; ++g) {
+            for (int g = 1; g < kRouterWarps; ++g) {
                 sum.x += part[g][lane].x;
                 sum.y += part[g][lane].y;
             }
