@@ -333,7 +333,37 @@ int flux_profile_read(flux_plan *plan, int32_t kind, double *total_ms, int64_t *
  *
  * flux_attn_combine: merges n_sets pieces laid out [n_sets][B][n_q_heads][...] (what an all-gather of the ranks'
  * pieces produces) into out bf16 [B][n_q_heads][head_dim]: m = max m_s, O = sum_s O_s 2^(m_s - m), l likewise,
- * out = O / l (a row whose pieces are all empty is zero). */
+ * out = O / l (a row whose pieces are all empty is zero).
+ *
+ * The exchange without a library call (the paper has no counterpart: it runs on one GPU).  Every rank owns a gather
+ * buffer gather_o fp32 [world][B][n_q_heads][head_dim], gather_ml fp32 [world][B][n_q_heads][2] and a flag array
+ * uint32 [world], zero-filled once, and knows the addresses of all ranks' three arrays as they are mapped on ITS
+ * GPU (its own plainly, the peers' through peer access / IPC or symmetric memory; on one NVSwitch domain: up to 8).
+ * flux_attn_decode_partial_push evaluates this rank's piece like flux_attn_decode_partial and its merge kernel
+ * stores every row straight into slot `rank` of every rank's gather buffer (plain stores to peer memory), then --
+ * after a system-scope fence by every CTA and a ticket among them -- sets entry `rank` of every rank's flag array to
+ * `seq` (release, system scope).  flux_attn_combine_wait is flux_attn_combine over this rank's own gather buffer,
+ * each CTA first waiting (acquire, system scope) until all `world` flags equal `seq`.  The wait is bounded:
+ * wait_cycles SM clock cycles (0 = about a second), then FLUX_STATUS_WAIT_EXPIRED and `out` is left unwritten.
+ * `seq` is any non-zero value that differs from the one used for the previous exchange through the same buffers
+ * (a step counter).  A rank may push exchange k + 1 into a buffer only when every rank has finished merging exchange
+ * k out of it: use one buffer set per layer (a rank cannot finish layer l + 1 of a step before every rank has
+ * merged layer l of it), or two sets alternately.  Both kernels of the pushing call and the waiting merge never wait
+ * for a kernel of the same GPU: the writers of the flags are kernels on other GPUs.  Errors: as the calls above;
+ * world outside [1, 8], rank outside [0, world), seq == 0 -> FLUX_E_INVALID_ARG. */
+typedef struct {
+    int32_t world, rank;
+    float *gather_o[8];      /* rank p's gather_o as addressable from this GPU */
+    float *gather_ml[8];
+    uint32_t *flags[8];
+} flux_peer_set;
+int flux_attn_decode_partial_push(flux_plan *plan, int32_t layer, int32_t B, const void *q, const void *const *k_caches,
+                                  const void *const *v_caches, const int32_t *ctx_len, const int32_t *key_begin /*device*/,
+                                  const int32_t *key_end /*device*/, const flux_peer_set *peers /*host*/, uint32_t seq,
+                                  void *stream);
+int flux_attn_combine_wait(flux_plan *plan, int32_t B, int32_t world, const float *gather_o, const float *gather_ml,
+                           const uint32_t *flags /*device, this rank's own*/, uint32_t seq, int64_t wait_cycles,
+                           void *out /*device bf16 [B][n_q_heads][head_dim]*/, void *stream);
 int flux_attn_decode_partial(flux_plan *plan, int32_t layer, int32_t B, const void *q, const void *const *k_caches,
                              const void *const *v_caches, const int32_t *ctx_len, const int32_t *key_begin,
                              const int32_t *key_end, float *part_o, float *part_ml, void *stream);

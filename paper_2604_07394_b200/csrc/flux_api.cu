@@ -107,6 +107,7 @@ WorkspaceLayout workspace_layout(const flux_config &c)
     w.router = off;       off = align_up(off + ((size_t)2 * c.n_q_heads * kHeadDim + 6 * kRouterMaxWidth) * sizeof(float), A);
     w.router_sync = off;  off = align_up(off + 8 * sizeof(uint32_t), A);
     w.tickets = off;      off = align_up(off + 2 * (size_t)kDecFusedMaxBatch * c.n_kv_heads * sizeof(uint32_t), A);
+    w.push_ticket = off;  off = align_up(off + 8 * sizeof(uint32_t), A);
     w.total = off;
     return w;
 }
@@ -641,9 +642,57 @@ int flux_attn_decode_partial(flux_plan *plan, int32_t layer, int32_t B, const vo
         return fail(FLUX_E_INVALID_ARG, "q / part_o must be 16-byte aligned, part_ml 8-byte aligned");
     if (!is_device_ptr(key_begin) || !is_device_ptr(key_end) || !is_device_ptr(part_o) || !is_device_ptr(part_ml))
         return fail(FLUX_E_INVALID_ARG, "key ranges and partial outputs must be device memory");
-    const DecPartial part = {key_begin, key_end, part_o, part_ml};
+    DecPartial part = {key_begin, key_end, part_o, part_ml, {}};
+    part.push.world = 0;
     return launch_decode(plan, layer, B, q, k_caches, v_caches, ctx_len, nullptr, (cudaStream_t)stream, nullptr, nullptr,
                          nullptr, &part);
+}
+
+int flux_attn_decode_partial_push(flux_plan *plan, int32_t layer, int32_t B, const void *q, const void *const *k_caches,
+                                  const void *const *v_caches, const int32_t *ctx_len, const int32_t *key_begin,
+                                  const int32_t *key_end, const flux_peer_set *peers, uint32_t seq, void *stream)
+{
+    int rc = check_batch_call(plan, layer, B);
+    if (rc) return rc;
+    if (!q || !k_caches || !v_caches || !ctx_len || !key_begin || !key_end || !peers)
+        return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    if (!aligned16(q)) return fail(FLUX_E_INVALID_ARG, "q must be 16-byte aligned");
+    if (!is_device_ptr(key_begin) || !is_device_ptr(key_end))
+        return fail(FLUX_E_INVALID_ARG, "key ranges must be device memory");
+    if (peers->world < 1 || peers->world > kMaxPeers || peers->rank < 0 || peers->rank >= peers->world)
+        return fail(FLUX_E_INVALID_ARG, "world=%d (1..%d) / rank=%d", peers->world, kMaxPeers, peers->rank);
+    if (seq == 0) return fail(FLUX_E_INVALID_ARG, "seq must not be 0 (the value of a cleared flag array)");
+    DecPartial part = {key_begin, key_end, nullptr, nullptr, {}};
+    part.push.world = peers->world;
+    part.push.rank = peers->rank;
+    part.push.seq = seq;
+    for (int p = 0; p < peers->world; ++p) {
+        if (!peers->gather_o[p] || !peers->gather_ml[p] || !peers->flags[p])
+            return fail(FLUX_E_INVALID_ARG, "peer %d: NULL pointer", p);
+        if (!aligned16(peers->gather_o[p]) || (((uintptr_t)peers->gather_ml[p]) & 7u) || (((uintptr_t)peers->flags[p]) & 3u))
+            return fail(FLUX_E_INVALID_ARG, "peer %d: gather_o must be 16-byte, gather_ml 8-byte, flags 4-byte aligned", p);
+        part.push.o[p] = peers->gather_o[p];
+        part.push.ml[p] = peers->gather_ml[p];
+        part.push.flags[p] = peers->flags[p];
+    }
+    return launch_decode(plan, layer, B, q, k_caches, v_caches, ctx_len, nullptr, (cudaStream_t)stream, nullptr, nullptr,
+                         nullptr, &part);
+}
+
+int flux_attn_combine_wait(flux_plan *plan, int32_t B, int32_t world, const float *gather_o, const float *gather_ml,
+                           const uint32_t *flags, uint32_t seq, int64_t wait_cycles, void *out, void *stream)
+{
+    int rc = need_plan(plan, true);
+    if (rc) return rc;
+    if (B < 1 || B > plan->cfg.max_batch) return fail(FLUX_E_CAPACITY, "B=%d outside [1, %d]", B, plan->cfg.max_batch);
+    if (world < 1 || world > kMaxPeers) return fail(FLUX_E_INVALID_ARG, "world=%d outside [1, %d]", world, kMaxPeers);
+    if (!gather_o || !gather_ml || !flags || !out) return fail(FLUX_E_INVALID_ARG, "NULL pointer");
+    if (!aligned16(gather_o) || !aligned16(out) || (((uintptr_t)gather_ml) & 7u) || (((uintptr_t)flags) & 3u))
+        return fail(FLUX_E_INVALID_ARG, "gather_o / out must be 16-byte, gather_ml 8-byte, flags 4-byte aligned");
+    if (seq == 0) return fail(FLUX_E_INVALID_ARG, "seq must not be 0");
+    if (wait_cycles < 0 || wait_cycles > 4000000000ll) return fail(FLUX_E_INVALID_ARG, "wait_cycles outside [0, 4e9]");
+    return launch_combine_sets(plan, gather_o, gather_ml, world, B * plan->cfg.n_q_heads, out, (cudaStream_t)stream, flags, seq,
+                               wait_cycles ? wait_cycles : 2000000000ll);
 }
 
 int flux_attn_combine(flux_plan *plan, int32_t B, int32_t n_sets, const float *part_o, const float *part_ml, void *out,
@@ -776,7 +825,7 @@ int flux_plan_status(flux_plan *plan, uint32_t *status_bits, void *stream)
         rc = check_cuda(cudaMemsetAsync((char *)plan->ws + plan->lay.router, 0,
                                         plan->lay.router_sync + 8 * sizeof(uint32_t) - plan->lay.router, st), "counter clear");
         if (!rc) rc = check_cuda(cudaMemsetAsync((char *)plan->ws + plan->lay.tickets, 0,
-                                                 2 * (size_t)kDecFusedMaxBatch * plan->cfg.n_kv_heads * sizeof(uint32_t), st), "counter clear");
+                                                 plan->lay.push_ticket + 8 * sizeof(uint32_t) - plan->lay.tickets, st), "counter clear");
         if (!rc) rc = check_cuda(cudaStreamSynchronize(st), "stream synchronize");
         if (rc) return rc;
     }

@@ -303,6 +303,34 @@ __global__ void __launch_bounds__(kDecWarps * 32, 1) decode_kernel(DecArgs a)
 // kernel itself), then the warps' results are merged through shared memory.
 constexpr int kCombWarps = 16;
 
+// Pushed pieces: channel d of the merged row of (request, head) `row` goes to slot push_rank of every gather buffer
+// -- this GPU's own and its peers', plain stores over NVLink -- and thread 0 adds (m, l).
+__device__ __forceinline__ void push_row(const DecArgs &a, size_t row, int d, float o, float m, float l)
+{
+    const size_t e = (size_t)a.push_rank * a.B * a.Hq + row;
+    for (int p = 0; p < a.push_world; ++p) {
+        a.push_o[p][e * kHeadDim + d] = o;
+        if (d == 0) *reinterpret_cast<float2 *>(a.push_ml[p] + e * 2) = make_float2(m, l);
+    }
+}
+// Called by every thread of every CTA of the merge launch once its stores are issued: the CTA that gets here last
+// tells every gather buffer's owner that this rank's piece is complete (flag = push_seq, released at system scope
+// after every CTA's stores, which each CTA fenced at system scope before it took its ticket).
+__device__ __forceinline__ void push_signal(const DecArgs &a)
+{
+    __threadfence_system();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned ticket;
+        asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;\n" : "=r"(ticket) : "l"(a.push_ticket) : "memory");
+        if (ticket == gridDim.x - 1) {
+            *a.push_ticket = 0u;
+            for (int p = 0; p < a.push_world; ++p)
+                asm volatile("st.release.sys.global.u32 [%0], %1;\n" ::"l"(a.push_flags[p] + a.push_rank), "r"(a.push_seq) : "memory");
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kCombWarps * 32) decode_combine_kernel(DecArgs a)
 {
     __shared__ float s_o[kCombWarps][kHeadDim];
@@ -318,6 +346,11 @@ __global__ void __launch_bounds__(kCombWarps * 32) decode_combine_kernel(DecArgs
     const int units = uend - ustart;
     float *pdst_o = a.pout_o ? a.pout_o + ((size_t)b * a.Hq + h) * kHeadDim : nullptr;
     if (units == 0) {  // inactive request (or, in a partial call, no key of the range is kept): nothing to add
+        if (a.push_world > 0) {
+            if (threadIdx.x < kHeadDim) push_row(a, (size_t)b * a.Hq + h, threadIdx.x, 0.f, kNegBig, 0.f);
+            push_signal(a);
+            return;
+        }
         if (threadIdx.x < kHeadDim) {
             if (pdst_o) pdst_o[threadIdx.x] = 0.f; else dst[threadIdx.x] = __float2bfloat16(0.f);
         }
@@ -386,7 +419,10 @@ __global__ void __launch_bounds__(kCombWarps * 32) decode_combine_kernel(DecArgs
         s_l[warp] = l;
     }
     __syncthreads();
-    if (threadIdx.x >= kHeadDim) return;
+    if (threadIdx.x >= kHeadDim) {
+        if (a.push_world > 0) push_signal(a);
+        return;
+    }
     const int d = threadIdx.x;
     float mm = kNegBig;
 #pragma unroll
@@ -398,7 +434,10 @@ __global__ void __launch_bounds__(kCombWarps * 32) decode_combine_kernel(DecArgs
         num += s_o[w][d] * sc;
         den += s_l[w] * sc;
     }
-    if (pdst_o) {   // partial call: the merged state itself (O unnormalised), for flux_attn_combine
+    if (a.push_world > 0) {   // pushed piece: the merged state goes straight into every rank's gather buffer
+        push_row(a, (size_t)b * a.Hq + h, d, num, mm, den);
+        push_signal(a);
+    } else if (pdst_o) {   // partial call: the merged state itself (O unnormalised), for flux_attn_combine
         pdst_o[d] = num;
         if (d == 0) *reinterpret_cast<float2 *>(a.pout_ml + ((size_t)b * a.Hq + h) * 2) = make_float2(mm, den);
     } else {
@@ -409,9 +448,36 @@ __global__ void __launch_bounds__(kCombWarps * 32) decode_combine_kernel(DecArgs
 // Merges n_sets partial evaluations of the same (request, query head) rows -- each (O unnormalised, m, l) over a
 // disjoint set of keys -- into the bf16 output: m = max m_s, O = sum O_s 2^(m_s - m), l likewise, out = O / l.
 // Sets are laid out [set][row]; one warp per row, four channels per lane, the sets taken in order.
-__global__ void __launch_bounds__(256) combine_sets_kernel(const float *__restrict__ po, const float *__restrict__ pml,
-                                                           int n_sets, int n_rows, __nv_bfloat16 *__restrict__ out)
+// With `flags` (flux_attn_combine_wait) the sets are pieces that other GPUs store into this buffer: set s is complete
+// once flags[s] holds `seq` (its owner releases the flag at system scope after its stores), and every CTA first waits for
+// all flags -- a bounded spin: the writers are kernels on other GPUs (or earlier launches on this one), which never wait
+// for this kernel -- and gives up with FLUX_STATUS_WAIT_EXPIRED, writing nothing, when the limit runs out.
+__global__ void __launch_bounds__(256) combine_sets_kernel(const float *po, const float *pml, int n_sets, int n_rows,
+                                                           __nv_bfloat16 *__restrict__ out, const uint32_t *flags, uint32_t seq,
+                                                           long long wait_cycles, uint32_t *status)
 {
+    if (flags != nullptr) {
+        __shared__ int s_ok;
+        if (threadIdx.x == 0) {
+            int ok = 1;
+            const long long t0 = clock64();
+            for (int s = 0; s < n_sets && ok; ++s) {
+                for (;;) {
+                    uint32_t v;
+                    asm volatile("ld.acquire.sys.global.u32 %0, [%1];\n" : "=r"(v) : "l"(flags + s) : "memory");
+                    if (v == seq) break;
+                    if (clock64() - t0 > wait_cycles) {
+                        atomicOr(status, FLUX_STATUS_WAIT_EXPIRED);
+                        ok = 0;
+                        break;
+                    }
+                }
+            }
+            s_ok = ok;
+        }
+        __syncthreads();
+        if (!s_ok) return;
+    }
     const int row = (int)((blockIdx.x * blockDim.x + threadIdx.x) >> 5), lane = threadIdx.x & 31;
     if (row >= n_rows) return;
     float m = kNegBig;
@@ -449,9 +515,11 @@ int decode_setup(flux_plan *p)
                       "cudaFuncSetAttribute(decode_kernel)");
 }
 
-int launch_combine_sets(flux_plan *p, const float *po, const float *pml, int n_sets, int n_rows, void *out, cudaStream_t st)
+int launch_combine_sets(flux_plan *p, const float *po, const float *pml, int n_sets, int n_rows, void *out, cudaStream_t st,
+                        const uint32_t *flags, uint32_t seq, long long wait_cycles)
 {
-    combine_sets_kernel<<<(n_rows + 7) / 8, 256, 0, st>>>(po, pml, n_sets, n_rows, (__nv_bfloat16 *)out);
+    combine_sets_kernel<<<(n_rows + 7) / 8, 256, 0, st>>>(po, pml, n_sets, n_rows, (__nv_bfloat16 *)out, flags, seq, wait_cycles,
+                                                         (uint32_t *)((char *)p->ws + p->lay.status));
     p->launches++;
     return check_cuda(cudaGetLastError(), "partial-set combine kernel launch");
 }
@@ -489,6 +557,16 @@ int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *con
     a.key_end = part ? part->key_end : nullptr;
     a.pout_o = part ? part->out_o : nullptr;
     a.pout_ml = part ? part->out_ml : nullptr;
+    a.push_world = part ? part->push.world : 0;
+    a.push_rank = part ? part->push.rank : 0;
+    a.push_seq = part ? part->push.seq : 0u;
+    for (int i = 0; i < kMaxPeers; ++i) {
+        const bool on = part && i < part->push.world;
+        a.push_o[i] = on ? part->push.o[i] : nullptr;
+        a.push_ml[i] = on ? part->push.ml[i] : nullptr;
+        a.push_flags[i] = on ? part->push.flags[i] : nullptr;
+    }
+    a.push_ticket = (uint32_t *)(ws + p->lay.push_ticket);
     const int fused_max = p->decode_kernel == FLUX_DECODE_SINGLE_LAUNCH ? kDecFusedMaxBatch
                           : p->decode_kernel == FLUX_DECODE_AUTO        ? kDecFusedAutoBatch : 0;
     if (head_mask == nullptr && part == nullptr && B <= fused_max && c.n_kv_heads <= kDecFusedMaxKvHeads)
@@ -648,6 +726,8 @@ extern "C" int flux_attn_decode_noalloc(const flux_config *cfg, int32_t layer, i
     a.overlap = 0;
     a.key_begin = a.key_end = nullptr;
     a.pout_o = a.pout_ml = nullptr;
+    a.push_world = 0;
+    a.push_ticket = nullptr;
     decode_kernel<<<nd->n_ctas, kDecWarps * 32, kDecSmemBytes, st>>>(a);
     rc = check_cuda(cudaGetLastError(), "decode kernel launch");
     if (rc) return rc;

@@ -43,6 +43,14 @@ struct DecArgs {
     // request, and where the merged (O, m, l) of every (request, query head) goes instead of the bf16 output
     const int32_t *key_begin, *key_end;
     float *pout_o, *pout_ml;
+    // pushed pieces (flux_attn_decode_partial_push): the merged piece of every (request, query head) goes into slot
+    // push_rank of each of push_world gather buffers (this GPU's own and its peers', all addresses valid here), then
+    // entry push_rank of each one's flag array is set to push_seq.  push_world == 0: off.
+    int push_world, push_rank;
+    uint32_t push_seq;
+    float *push_o[kMaxPeers], *push_ml[kMaxPeers];
+    uint32_t *push_flags[kMaxPeers];
+    uint32_t *push_ticket;      // workspace counter: CTAs of the merge launch that have stored their rows (zero between launches)
 };
 
 // What one request contributes to this layer's launch.

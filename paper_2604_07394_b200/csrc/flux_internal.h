@@ -19,6 +19,7 @@ constexpr int kDecTile = 16;        // tokens per pipeline stage of one warp
 constexpr int kDecStages = 3;       // cp.async stages per warp
 constexpr int kDecStageBytes = kDecTile * kRowBytes * 2;  // K tile + V tile
 constexpr int kDecMaxCtas = 512;    // upper bound used to size the workspace
+constexpr int kMaxPeers = 8;        // GPUs a decode step's keys can be spread over (one NVSwitch domain)
 constexpr int kMaxBatch = 1024;     // prefix tables live in shared memory
 constexpr int kDecFusedMaxBatch = 32;   // largest batch the single-launch decode kernel takes
 constexpr int kDecFusedAutoBatch = 32;  // largest batch it is chosen for by default
@@ -40,6 +41,7 @@ struct WorkspaceLayout {
     size_t host_o;       // bf16  [max_batch][Hq][D]
     size_t router;       // fp32 [2*Hq*D] pooled descriptor, then uint64 [3][kRouterMaxWidth] hidden activations (value | launch number << 32)
     size_t router_sync;  // uint32 [8]: barrier counter and exit ticket of the router front end (zero between launches), its launch number
+    size_t push_ticket;  // uint32 [8]: CTAs of a pushing merge launch that have stored their rows (zero between launches)
     size_t tickets;      // uint32 [2][kDecFusedMaxBatch][Hkv] arrival / helper counters of the single-launch decode (zero between launches)
     size_t total;
     int64_t slots;
@@ -109,15 +111,23 @@ int launch_kv_retain(flux_plan *p, int layer, int req, const void *k_src, const 
 // head_mask non-NULL: per-KV-head modes [B][Hkv] instead of the routed layer mask (flux_attn_decode_heads)
 // part non-NULL: evaluate only the keys [key_begin[b], key_end[b]) and write the merged (O, m, l) of every
 // (request, query head) to out_o / out_ml instead of the bf16 output (flux_attn_decode_partial)
+struct DecPush {              // where a pushed piece goes (flux_attn_decode_partial_push); world == 0: nowhere
+    int world, rank;
+    uint32_t seq;
+    float *o[kMaxPeers], *ml[kMaxPeers];
+    uint32_t *flags[kMaxPeers];
+};
 struct DecPartial {
     const int32_t *key_begin, *key_end;
     float *out_o, *out_ml;
+    DecPush push;
 };
 int launch_decode(flux_plan *p, int layer, int B, const void *q, const void *const *k_caches,
                   const void *const *v_caches, const int32_t *ctx_len, void *out,
                   cudaStream_t st, const void *k_new = nullptr, const void *v_new = nullptr,
                   const uint8_t *head_mask = nullptr, const DecPartial *part = nullptr);
-int launch_combine_sets(flux_plan *p, const float *po, const float *pml, int n_sets, int n_rows, void *out, cudaStream_t st);
+int launch_combine_sets(flux_plan *p, const float *po, const float *pml, int n_sets, int n_rows, void *out, cudaStream_t st,
+                        const uint32_t *flags = nullptr, uint32_t seq = 0, long long wait_cycles = 0);
 int launch_prefill(flux_plan *p, int layer, int req, const void *q, const void *k, const void *v,
                    int q_start, int Nq, void *out, cudaStream_t st);
 // bracket a dominant-kernel launch with events when profiling is on

@@ -44,7 +44,7 @@ FLUX_KV_COMPACT_SA = 1
 EXPORTS = [
     "flux_plan_create", "flux_plan_destroy", "flux_workspace_size", "flux_plan_set_workspace",
     "flux_router_apply", "flux_router_forward", "flux_attn_prefill", "flux_attn_prefill_blocks", "flux_kv_retain", "flux_kv_append",
-    "flux_attn_decode", "flux_attn_decode_heads", "flux_attn_decode_partial", "flux_attn_combine", "flux_attn_decode_step", "flux_attn_decode_noalloc", "flux_attn_decode_host", "flux_attn_prefill_host", "flux_plan_status",
+    "flux_attn_decode", "flux_attn_decode_heads", "flux_attn_decode_partial", "flux_attn_combine", "flux_attn_decode_partial_push", "flux_attn_combine_wait", "flux_attn_decode_step", "flux_attn_decode_noalloc", "flux_attn_decode_host", "flux_attn_prefill_host", "flux_plan_status",
     "flux_debug_dispatch", "flux_debug_touched", "flux_debug_decode_kernel", "flux_plan_set_launch_overlap", "flux_debug_wait_probe", "flux_profile_enable", "flux_profile_read", "flux_launch_count", "flux_last_error", "flux_version",
 ]
 
@@ -65,6 +65,13 @@ class FluxRouterWeights(ctypes.Structure):
         ("w_enc2", ctypes.c_void_p), ("b_enc2", ctypes.c_void_p),
         ("w_head1", ctypes.c_void_p), ("b_head1", ctypes.c_void_p),
         ("w_head2", ctypes.c_void_p), ("b_head2", ctypes.c_void_p),
+    ]
+
+
+class PeerSet(ctypes.Structure):
+    _fields_ = [
+        ("world", ctypes.c_int32), ("rank", ctypes.c_int32),
+        ("gather_o", ctypes.c_void_p * 8), ("gather_ml", ctypes.c_void_p * 8), ("flags", ctypes.c_void_p * 8),
     ]
 
 
@@ -102,6 +109,8 @@ def load():
     L.flux_attn_decode.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode_partial.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp]
     L.flux_attn_combine.argtypes = [vp, i32, i32, vp, vp, vp, vp]
+    L.flux_attn_decode_partial_push.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, ctypes.c_uint32, vp]
+    L.flux_attn_combine_wait.argtypes = [vp, i32, i32, vp, vp, vp, ctypes.c_uint32, ctypes.c_int64, vp, vp]
     L.flux_attn_decode_heads.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.flux_attn_decode_noalloc.argtypes = [cfgp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -270,6 +279,24 @@ class Plan:
         if out is None:
             out = torch.empty((B, self.cfg.n_q_heads, 128), dtype=torch.bfloat16, device=self.device)
         _check(load().flux_attn_combine(self._h, B, n_sets, _ptr(part_o), _ptr(part_ml), _ptr(out), _stream()))
+        return out
+
+    def flux_attn_decode_partial_push(self, layer, B, q, k_caches, v_caches, ctx_len, key_begin, key_end, rank, gather_o, gather_ml, flags, seq):
+        """This rank's piece stored straight into slot `rank` of every rank's gather buffer; gather_o / gather_ml / flags:
+        one tensor per rank (fp32 [world][B][Hq][D], fp32 [world][B][Hq][2], int32 or uint32 [world]), addressable from this GPU."""
+        ps = PeerSet()
+        ps.world, ps.rank = len(gather_o), rank
+        for p in range(ps.world):
+            ps.gather_o[p], ps.gather_ml[p], ps.flags[p] = _ptr(gather_o[p]), _ptr(gather_ml[p]), _ptr(flags[p])
+        _check(load().flux_attn_decode_partial_push(self._h, layer, B, _ptr(q), _ptr(k_caches), _ptr(v_caches), _ptr(ctx_len),
+                                                    _ptr(key_begin), _ptr(key_end), ctypes.byref(ps), seq, _stream()))
+
+    def flux_attn_combine_wait(self, B, gather_o, gather_ml, flags, seq, out=None, wait_cycles=0):
+        """Waits (bounded) until every rank's flag equals seq, then merges this rank's gather buffer -> out bf16 [B][Hq][D]."""
+        if out is None:
+            out = torch.empty((B, self.cfg.n_q_heads, 128), dtype=torch.bfloat16, device=self.device)
+        _check(load().flux_attn_combine_wait(self._h, B, int(gather_o.shape[0]), _ptr(gather_o), _ptr(gather_ml), _ptr(flags), seq,
+                                             wait_cycles, _ptr(out), _stream()))
         return out
 
     def flux_attn_decode_heads(self, B, q, k_caches, v_caches, ctx_len, head_mask, out=None):
