@@ -5,7 +5,9 @@ computes the piece with ``flux_attn_decode_partial``, the pieces are exchanged w
 (``B * n_q_heads * 130`` floats per rank and layer) and every rank merges them with
 ``flux_attn_combine``.  This module only cuts ranges and moves pieces; it holds no attention
 arithmetic.  The exchange is a plain ``torch.distributed`` all-gather (NCCL on GPUs, gloo in the CPU
-tests).
+tests).  The second form of the exchange needs no collective: ``flux_attn_decode_partial_push`` stores a
+rank's piece into every rank's gather buffer and raises a flag, ``flux_attn_combine_wait`` waits for the
+flags; ``exchange_seq`` and ``buffer_set`` give the sequence number and the buffer set that form uses.
 """
 from __future__ import annotations
 
@@ -41,3 +43,20 @@ def all_gather_pieces(dist, part_o: torch.Tensor, part_ml: torch.Tensor, group=N
     dist.all_gather_into_tensor(po, part_o.contiguous(), group=group)
     dist.all_gather_into_tensor(pml, part_ml.contiguous(), group=group)
     return po.view((world,) + tuple(part_o.shape)), pml.view((world,) + tuple(part_ml.shape))
+
+
+def exchange_seq(step: int) -> int:
+    """Sequence number of decode step ``step`` (0, 1, 2, ...) for the pushed exchange: never 0 (a cleared flag
+    array holds zeros), different for consecutive steps, inside 32 bits."""
+    assert step >= 0
+    return step % 0xFFFFFFFF + 1
+
+
+def buffer_set(step: int, layer: int, n_layers: int) -> int:
+    """Which gather buffer set (gather_o, gather_ml, flags) the exchange of (step, layer) goes through.  A set may
+    be written again only when every rank has merged the previous exchange out of it.  With at least two layers,
+    one set per layer is enough: a rank cannot push layer ``l`` of the next step before it has finished this
+    step, hence not before every rank has pushed -- and so merged layer ``l`` of -- this step's later layers.
+    A single-layer stack alternates two sets."""
+    assert 0 <= layer < n_layers
+    return layer if n_layers >= 2 else step % 2

@@ -26,3 +26,11 @@ def test_key_ranges_hand_typed():
     r = keysplit.key_ranges([100, 5], 2, 16)
     assert r.tolist() == [[[0, 64], [0, 5]], [[64, 100], [5, 5]]]        # 50 rounded up to 64; 2.5 -> 16, clipped to 5
     assert keysplit.key_ranges([48], 3, 16).tolist() == [[[0, 16]], [[16, 32]], [[32, 48]]]
+
+
+def test_exchange_sequence_numbers_and_buffer_sets():
+    seqs = [keysplit.exchange_seq(t) for t in range(6)] + [keysplit.exchange_seq(0xFFFFFFFE), keysplit.exchange_seq(0xFFFFFFFF)]
+    assert seqs[:3] == [1, 2, 3] and all(0 < s <= 0xFFFFFFFF for s in seqs)
+    assert all(a != b for a, b in zip(seqs, seqs[1:]))                   # also across the wrap: 0xFFFFFFFF then 1
+    assert [keysplit.buffer_set(t, l, 3) for t in range(2) for l in range(3)] == [0, 1, 2, 0, 1, 2]
+    assert [keysplit.buffer_set(t, 0, 1) for t in range(4)] == [0, 1, 0, 1]
